@@ -1,0 +1,291 @@
+/*
+ * PrefixKV CPU oracle -- TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, single-threaded restatement of what the PrefixKV hot path
+ * computes, written from the paper's definitions.  It exists so that the CUDA
+ * library can be checked element by element; it shares no code, header, table
+ * or helper with that library, and nothing in the product may call it.
+ *
+ * Floating-point work is done in fp64 (inputs arrive as fp32 values, which
+ * hold bf16 exactly); the two places where an fp32 value decides an integer
+ * (the sort key and the fixed-point weight) use the fp32 score itself.
+ *
+ * Notation follows the paper: L layers, H heads, N prompt tokens, D head dim,
+ * I_l^n importance, s_l^j sorted indices, P_l^o cumulative priority, p the
+ * information-retention ratio, R_l retained ratio (here the integer R_l * N).
+ *
+ * Pins (tests/test_oracle_*.py): harmonic-number closed form and softmax
+ * column sums via a library softmax for the score; library stable sort for the
+ * order; exact rational arithmetic for the cumulative weights; brute-force
+ * enumeration of every breakpoint of p and a hand-worked example for the
+ * search; library dense attention for decode.  Unpinned: nothing in this file
+ * (iteration counts and model quality reported by the paper are not
+ * reproducible without its data and are not claimed).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum {
+    ORC_OK = 0,
+    ORC_BAD_SCORE = 1,        /* NaN, inf or negative importance          */
+    ORC_RANGE = 2,            /* fixed-point total does not fit in 2^53   */
+    ORC_BUDGET_TOO_SMALL = 3, /* budget < L: one row per layer is minimal */
+    ORC_BAD_LENGTH = 4        /* given length outside [1, N]              */
+};
+
+/* ------------------------------------------------------------------------
+ * Importance score, Sec. 3.2: a_l^{i,m,n} is the causal softmax over keys
+ * j <= m of scale * (q^{i,m} . k^{i,j}); I_l^n averages over heads i the sum
+ * over queries m of a_l^{i,m,n}.  (The printed formula has no scale; scale = 1
+ * reproduces it.  The max subtraction leaves the quotient unchanged.)
+ *
+ * q, k: [H][N][D] fp32, one layer of one sample.  out_f32[N] is I rounded once
+ * to fp32; out_f64[N] (may be NULL) is the unrounded value.
+ * ---------------------------------------------------------------------- */
+void orc_score_layer(const float *q, const float *k, int H, int N, int D,
+                     double scale, float *out_f32, double *out_f64)
+{
+    double *col = (double *)calloc((size_t)N, sizeof(double));
+    double *s = (double *)malloc((size_t)N * sizeof(double));
+    for (int i = 0; i < H; ++i) {
+        const float *qh = q + (size_t)i * N * D;
+        const float *kh = k + (size_t)i * N * D;
+        for (int m = 0; m < N; ++m) {
+            double mx = -INFINITY;
+            for (int j = 0; j <= m; ++j) {
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d)
+                    dot += (double)qh[(size_t)m * D + d] * (double)kh[(size_t)j * D + d];
+                s[j] = scale * dot;
+                if (s[j] > mx) mx = s[j];
+            }
+            double z = 0.0;
+            for (int j = 0; j <= m; ++j) z += exp(s[j] - mx);
+            for (int j = 0; j <= m; ++j) col[j] += exp(s[j] - mx) / z;
+        }
+    }
+    for (int n = 0; n < N; ++n) {
+        double v = col[n] / (double)H;
+        if (out_f64) out_f64[n] = v;
+        out_f32[n] = (float)v;
+    }
+    free(s);
+    free(col);
+}
+
+/* ------------------------------------------------------------------------
+ * Priority sequence, Sec. 3.2: indices sorted by importance, descending.
+ * Ties are broken by position ascending (the paper is silent; this makes the
+ * order unique).  -0.0 and +0.0 compare equal, as IEEE says.  Insertion sort:
+ * slow, stable, obviously right.
+ * ---------------------------------------------------------------------- */
+static int precedes(const float *I, int32_t a, int32_t b)
+{
+    if (I[a] > I[b]) return 1;
+    if (I[a] < I[b]) return 0;
+    return a < b;
+}
+
+void orc_sort_desc(const float *I, int N, int32_t *order)
+{
+    for (int n = 0; n < N; ++n) {
+        int32_t cur = n;
+        int j = n;
+        while (j > 0 && precedes(I, cur, order[j - 1])) {
+            order[j] = order[j - 1];
+            --j;
+        }
+        order[j] = cur;
+    }
+}
+
+/* ------------------------------------------------------------------------
+ * Cumulative priority, Sec. 3.2: P_l^o = sum_{j <= oN} of the normalised
+ * importance of s_l^j.  The normaliser is never divided out: P >= p is tested
+ * as cum >= p * total.  Sums are kept in 2^-32 fixed point so that they do not
+ * depend on summation order: w = round-half-even(I * 2^32) (the product is
+ * exact in fp64), cum[j] = w_0 + ... + w_j in uint64.
+ * Returns ORC_BAD_SCORE / ORC_RANGE when the inputs break the preconditions.
+ * ---------------------------------------------------------------------- */
+int orc_cumulative(const float *I, const int32_t *order, int N, uint64_t *cum)
+{
+    uint64_t run = 0;
+    for (int j = 0; j < N; ++j) {
+        float v = I[order[j]];
+        if (!(v >= 0.0f) || isinf(v)) return ORC_BAD_SCORE;
+        double scaled = ldexp((double)v, 32);
+        if (scaled >= 9007199254740992.0) return ORC_RANGE;
+        uint64_t w = (uint64_t)llrint(scaled); /* default rounding: half-even */
+        run += w;
+        if (run >= (1ull << 53)) return ORC_RANGE;
+        cum[j] = run;
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * Retained length of one layer for a given p, Sec. 3.3:
+ * R_l = min{ o | P_l^o >= p }, returned as the row count R_l * N in [1, N].
+ * p >= 1 keeps everything by definition; otherwise the threshold is
+ * theta = ceil(p * total) and the answer is the first 1-based j with
+ * cum[j] >= theta.
+ * ---------------------------------------------------------------------- */
+int32_t orc_length_for_p(const uint64_t *cum, int N, double p)
+{
+    if (p >= 1.0) return N;
+    double total = (double)cum[N - 1];
+    volatile double prod = p * total; /* one rounded multiply, no contraction */
+    uint64_t theta = (uint64_t)ceil(prod);
+    int32_t below = 0;
+    for (int j = 0; j < N; ++j)
+        if (cum[j] < theta) ++below;
+    int32_t n = 1 + below;
+    if (n > N) n = N;
+    return n;
+}
+
+static int64_t total_length(const uint64_t *cum, int L, int N, double p, int32_t *len)
+{
+    int64_t S = 0;
+    for (int l = 0; l < L; ++l) {
+        len[l] = orc_length_for_p(cum + (size_t)l * N, N, p);
+        S += len[l];
+    }
+    return S;
+}
+
+/* ------------------------------------------------------------------------
+ * Binary search for p, Algorithm 1 and Eq. 1, with the budget as an integer
+ * number of rows summed over layers (r * L * N).  delta = S(p) - budget.
+ * delta == 0 returns p; delta < 0 raises p1; otherwise lowers p2.  The printed
+ * loop condition never becomes false, so the search also stops when the
+ * interval is no wider than tol, after max_iters evaluations, or when fp64
+ * cannot split the interval further; it then returns the lower end p1, whose
+ * configuration never exceeds the budget.  A one-sided threshold on delta
+ * (0 <= budget - S <= slack) is the paper's "small threshold for delta".
+ *
+ * cum: [L][N].  Outputs: len[L], *p_out, *iters_out (evaluations of S at a
+ * midpoint).  Returns ORC_BUDGET_TOO_SMALL if budget < L.
+ * ---------------------------------------------------------------------- */
+int orc_search(const uint64_t *cum, int L, int N, int64_t budget, double tol,
+               int32_t max_iters, int64_t slack, int32_t *len, double *p_out,
+               int32_t *iters_out)
+{
+    *iters_out = 0;
+    if (budget < (int64_t)L) {
+        *p_out = 0.0;
+        for (int l = 0; l < L; ++l) len[l] = 1;
+        return ORC_BUDGET_TOO_SMALL;
+    }
+    if ((int64_t)L * (int64_t)N <= budget) {
+        total_length(cum, L, N, 1.0, len);
+        *p_out = 1.0;
+        return ORC_OK;
+    }
+    double p1 = 0.0, p2 = 1.0;
+    int32_t iters = 0;
+    for (;;) {
+        double p = (p1 + p2) / 2.0;
+        if (p == p1 || p == p2 || iters == max_iters || p2 - p1 <= tol) break;
+        int64_t S = total_length(cum, L, N, p, len);
+        ++iters;
+        int64_t delta = S - budget;
+        if (delta == 0 || (delta < 0 && -delta <= slack)) {
+            *p_out = p;
+            *iters_out = iters;
+            return ORC_OK;
+        }
+        if (delta < 0) p1 = p; else p2 = p;
+    }
+    total_length(cum, L, N, p1, len);
+    *p_out = p1;
+    *iters_out = iters;
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * Lengths given from outside (offline configuration, Sec. 3.3 last paragraph,
+ * or the uniform R_j = r of Sec. 3.2): validate only.
+ * ---------------------------------------------------------------------- */
+int orc_check_lengths(const int32_t *len_in, int L, int N)
+{
+    for (int l = 0; l < L; ++l)
+        if (len_in[l] < 1 || len_in[l] > N) return ORC_BAD_LENGTH;
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * Compression after prefilling, Sec. 3.1 / Fig. 2(a): keep the first `len`
+ * entries of the priority sequence, the same set for every head.  kept[] lists
+ * the retained positions in ascending position; rows are copied in that order.
+ * src: [H][N][D]; dst: [len][H][D].
+ * ---------------------------------------------------------------------- */
+void orc_retained_positions(const int32_t *order, int N, int32_t len, int32_t *kept)
+{
+    unsigned char *flag = (unsigned char *)calloc((size_t)N, 1);
+    for (int j = 0; j < len; ++j) flag[order[j]] = 1;
+    int32_t w = 0;
+    for (int n = 0; n < N; ++n)
+        if (flag[n]) kept[w++] = n;
+    free(flag);
+}
+
+void orc_gather_rows(const float *src, int H, int N, int D, const int32_t *kept,
+                     int32_t len, float *dst)
+{
+    for (int r = 0; r < len; ++r)
+        for (int h = 0; h < H; ++h)
+            memcpy(dst + ((size_t)r * H + h) * D,
+                   src + ((size_t)h * N + kept[r]) * D, (size_t)D * sizeof(float));
+}
+
+/* ------------------------------------------------------------------------
+ * Decode attention, Sec. 3.1: the newest token's query attends to every cached
+ * row (its own key/value row has already been appended).
+ * kc, vc: [rows][H][D]; q: [H][D]; out: [H][D] in fp64.
+ * ---------------------------------------------------------------------- */
+void orc_decode_attn(const float *q, const float *kc, const float *vc, int rows,
+                     int H, int D, double scale, double *out)
+{
+    double *s = (double *)malloc((size_t)rows * sizeof(double));
+    for (int h = 0; h < H; ++h) {
+        double mx = -INFINITY;
+        for (int r = 0; r < rows; ++r) {
+            double dot = 0.0;
+            for (int d = 0; d < D; ++d)
+                dot += (double)q[(size_t)h * D + d] * (double)kc[((size_t)r * H + h) * D + d];
+            s[r] = scale * dot;
+            if (s[r] > mx) mx = s[r];
+        }
+        double z = 0.0;
+        for (int r = 0; r < rows; ++r) z += exp(s[r] - mx);
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int r = 0; r < rows; ++r)
+                acc += (exp(s[r] - mx) / z) * (double)vc[((size_t)r * H + h) * D + d];
+            out[(size_t)h * D + d] = acc;
+        }
+    }
+    free(s);
+}
+
+/* ------------------------------------------------------------------------
+ * Lorenz curve / Gini coefficient of a layer's priority sequence, Sec. 3.2
+ * (Fig. 3): area between the equality line and the curve, doubled, with the
+ * curve drawn over the ascending importance order (trapezoids).
+ * ---------------------------------------------------------------------- */
+double orc_gini(const float *I, const int32_t *order, int N)
+{
+    double total = 0.0;
+    for (int n = 0; n < N; ++n) total += (double)I[n];
+    if (!(total > 0.0)) return 0.0;
+    double area = 0.0, run = 0.0;
+    for (int j = N - 1; j >= 0; --j) { /* ascending = reverse of the priority order */
+        double prev = run;
+        run += (double)I[order[j]] / total;
+        area += (prev + run) / (2.0 * N);
+    }
+    return 1.0 - 2.0 * area;
+}

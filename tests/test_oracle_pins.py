@@ -1,0 +1,402 @@
+"""Pins for the CPU oracle: closed forms, library routines, exact arithmetic,
+brute force and a hand-worked example.  None of these re-type the oracle's own
+loops; each is chosen so that a plausible slip (sign, index, transposed operand,
+missing term, wrong tie-break or rounding) fails."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --------------------------------------------------------------------------
+# Importance score (Sec. 3.2)
+# --------------------------------------------------------------------------
+def _softmax_colsum_library(q, k, scale):
+    """Column sums of the causal softmax via torch.softmax on a masked matrix."""
+    H, N, D = q.shape
+    qt = torch.from_numpy(q).double()
+    kt = torch.from_numpy(k).double()
+    logits = scale * qt @ kt.transpose(1, 2)                      # [H, m, n]
+    mask = torch.ones(N, N, dtype=torch.bool).tril()              # n <= m
+    logits = logits.masked_fill(~mask, float("-inf"))
+    a = torch.softmax(logits, dim=-1)
+    return a.sum(dim=1).mean(dim=0).numpy()                       # sum over m, mean over heads
+
+
+@pytest.mark.parametrize("H,N,D,scale", [(3, 37, 8, 0.7), (2, 64, 16, 1.0), (1, 5, 4, 2.5)])
+def test_score_matches_library_softmax(H, N, D, scale):
+    rng = np.random.default_rng(H * 100 + N)
+    q = rng.standard_normal((H, N, D)).astype(np.float32)
+    k = rng.standard_normal((H, N, D)).astype(np.float32)
+    f32, f64 = oracle.score_layer(q, k, scale, want_f64=True)
+    ref = _softmax_colsum_library(q, k, scale)
+    np.testing.assert_allclose(f64, ref, rtol=1e-12, atol=1e-14)
+    np.testing.assert_array_equal(f32, ref.astype(np.float32))
+    # swapping the operands must not give the same answer (transposition check)
+    swapped = oracle.score_layer(k, q, scale)
+    assert np.abs(swapped - f32).max() > 1e-3
+
+
+def test_score_zero_query_is_harmonic():
+    """Q = 0 makes every causal row uniform: a^{m,n} = 1/m, so
+    I^n = H_N - H_{n-1} (1-based n), for any head count."""
+    H, N, D = 3, 50, 4
+    rng = np.random.default_rng(1)
+    q = np.zeros((H, N, D), np.float32)
+    k = rng.standard_normal((H, N, D)).astype(np.float32)
+    _, f64 = oracle.score_layer(q, k, 1.0, want_f64=True)
+    harm = [Fraction(0)]
+    for i in range(1, N + 1):
+        harm.append(harm[-1] + Fraction(1, i))
+    ref = np.array([float(harm[N] - harm[n]) for n in range(N)])
+    np.testing.assert_allclose(f64, ref, rtol=1e-13)
+    # same with scale = 0 and arbitrary Q
+    q2 = rng.standard_normal((H, N, D)).astype(np.float32)
+    _, g64 = oracle.score_layer(q2, k, 0.0, want_f64=True)
+    np.testing.assert_allclose(g64, ref, rtol=1e-13)
+
+
+def test_score_invariants():
+    H, N, D = 4, 48, 8
+    rng = np.random.default_rng(2)
+    q = rng.standard_normal((H, N, D)).astype(np.float32)
+    k = rng.standard_normal((H, N, D)).astype(np.float32)
+    _, I = oracle.score_layer(q, k, 0.9, want_f64=True)
+    # every causal softmax row sums to one, so the scores sum to N
+    assert abs(I.sum() - N) < 1e-9 * N
+    # first key is seen by every query and alone by the first: I^1 >= 1
+    assert I[0] >= 1.0
+    # last key is seen only by the last query: I^N = mean_h a^{N,N}
+    ref = _softmax_colsum_library(q, k, 0.9)
+    assert abs(I[-1] - ref[-1]) < 1e-14
+    # the head mean does not depend on head order
+    perm = np.array([2, 0, 3, 1])
+    _, Ip = oracle.score_layer(q[perm], k[perm], 0.9, want_f64=True)
+    np.testing.assert_allclose(Ip, I, rtol=1e-13)
+    # adding one vector to every key shifts each row's logits by a constant
+    kq = np.round(k * 1024) / np.float32(1024)          # so that k + 0.5 is exact in fp32
+    c = np.full((1, 1, D), 0.5, np.float32)
+    _, I0 = oracle.score_layer(q, kq, 0.9, want_f64=True)
+    _, Is = oracle.score_layer(q, kq + c, 0.9, want_f64=True)
+    np.testing.assert_allclose(Is, I0, rtol=1e-11)
+    # head mean, not head sum: duplicating the heads changes nothing
+    _, Id = oracle.score_layer(np.concatenate([q, q]), np.concatenate([k, k]), 0.9, want_f64=True)
+    np.testing.assert_allclose(Id, I, rtol=1e-13)
+
+
+def test_score_single_token():
+    q = np.full((2, 1, 4), 3.0, np.float32)
+    assert oracle.score_layer(q, q, 1.0)[0] == 1.0
+
+
+# --------------------------------------------------------------------------
+# Priority sequence (Sec. 3.2)
+# --------------------------------------------------------------------------
+def test_sort_matches_library_and_tie_break():
+    rng = np.random.default_rng(3)
+    for N in (1, 2, 17, 300):
+        s = rng.random(N).astype(np.float32)
+        s[rng.integers(0, N, N // 3 + 1)] = s[rng.integers(0, N, N // 3 + 1)]   # ties
+        ref = sorted(range(N), key=lambda n: (-float(s[n]), n))
+        np.testing.assert_array_equal(oracle.sort_desc(s), ref)
+    np.testing.assert_array_equal(oracle.sort_desc(np.ones(9, np.float32)), np.arange(9))
+    np.testing.assert_array_equal(oracle.sort_desc(np.arange(9, dtype=np.float32)), np.arange(9)[::-1])
+    # -0.0 and +0.0 are one value: position decides
+    z = np.array([0.0, -0.0, 1.0, -0.0, 0.0], np.float32)
+    np.testing.assert_array_equal(oracle.sort_desc(z), [2, 0, 1, 3, 4])
+
+
+# --------------------------------------------------------------------------
+# Cumulative priority in 2^-32 fixed point (Sec. 3.2)
+# --------------------------------------------------------------------------
+def _round_half_even(fr: Fraction) -> int:
+    fl = fr.numerator // fr.denominator
+    rem = fr - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        return fl + 1
+    return fl
+
+
+def test_cumulative_exact_arithmetic():
+    rng = np.random.default_rng(4)
+    N = 200
+    s = np.exp(rng.standard_normal(N) * 3 - 8).astype(np.float32)
+    s[:4] = [2.0 ** -33, 3 * 2.0 ** -33, 5 * 2.0 ** -33, 2.0 ** -34]      # halves: 0, 2, 2, 0
+    order = oracle.sort_desc(s)
+    cum, st = oracle.cumulative(s, order)
+    assert st == oracle.OK
+    run, ref = 0, []
+    for j in order:
+        run += _round_half_even(Fraction(float(s[j])) * 2 ** 32)
+        ref.append(run)
+    assert [int(c) for c in cum] == ref
+    assert all(int(cum[i]) <= int(cum[i + 1]) for i in range(N - 1))
+    # the total does not depend on the order of summation
+    rev, _ = oracle.cumulative(s, order[::-1].copy())
+    assert int(rev[-1]) == int(cum[-1])
+    w = {float(s[i]): _round_half_even(Fraction(float(s[i])) * 2 ** 32) for i in range(4)}
+    assert [w[float(s[i])] for i in range(4)] == [0, 2, 2, 0]
+
+
+def test_cumulative_rejects_bad_scores():
+    for bad in (float("nan"), float("inf"), -1.0):
+        s = np.array([1.0, bad, 0.5], np.float32)
+        _, st = oracle.cumulative(s, np.array([0, 1, 2], np.int32))
+        assert st == oracle.BAD_SCORE
+    s = np.array([2.0 ** 22, 1.0], np.float32)            # 2^54 in fixed point
+    _, st = oracle.cumulative(s, np.array([0, 1], np.int32))
+    assert st == oracle.RANGE
+
+
+# --------------------------------------------------------------------------
+# Retained length for a given p (Sec. 3.3)
+# --------------------------------------------------------------------------
+def test_length_rule_special_cases():
+    N = 64
+    ones = np.ones(N, np.float32)
+    cum, _ = oracle.cumulative(ones, np.arange(N, dtype=np.int32))
+    for p in (0.0, 1e-9, 0.1, 0.25, 0.3, 0.5, 0.77, 0.999):
+        assert oracle.length_for_p(cum, p) == max(1, math.ceil(p * N)), p
+    assert oracle.length_for_p(cum, 1.0) == N and oracle.length_for_p(cum, 1.5) == N
+    onehot = np.zeros(N, np.float32); onehot[7] = 3.0
+    order = oracle.sort_desc(onehot)
+    cum, _ = oracle.cumulative(onehot, order)
+    assert order[0] == 7
+    for p in (0.0, 0.3, 0.999999):
+        assert oracle.length_for_p(cum, p) == 1
+    assert oracle.length_for_p(cum, 1.0) == N
+    # equality at the threshold counts as reached ("larger than or equal to")
+    s = np.array([0.5, 0.25, 0.25], np.float32)
+    cum, _ = oracle.cumulative(s, np.arange(3, dtype=np.int32))
+    assert oracle.length_for_p(cum, 0.5) == 1
+    assert oracle.length_for_p(cum, np.nextafter(0.5, 1.0)) == 2
+    assert oracle.length_for_p(cum, 0.75) == 2
+    # monotone in p
+    rng = np.random.default_rng(5)
+    s = rng.random(100).astype(np.float32)
+    cum, _ = oracle.cumulative(s, oracle.sort_desc(s))
+    lens = [oracle.length_for_p(cum, p) for p in np.linspace(0, 1, 501)]
+    assert lens == sorted(lens) and lens[0] == 1 and lens[-1] == 100
+
+
+# --------------------------------------------------------------------------
+# Binary search (Algorithm 1, Eq. 1)
+# --------------------------------------------------------------------------
+def _length_exact(cum_row, p: float) -> int:
+    """The length rule re-derived with Python integers (no oracle code)."""
+    N = len(cum_row)
+    if p >= 1.0:
+        return N
+    theta = math.ceil(p * float(int(cum_row[-1])))
+    return min(N, 1 + sum(1 for c in cum_row if int(c) < theta))
+
+
+def _brute_force_config(cum, budget):
+    """Largest feasible configuration by trying every breakpoint of S(p).
+
+    S only changes where p * total crosses a cumulative value, so the fp64
+    numbers around each cum/total are the only places the answer can change."""
+    L, N = cum.shape
+    cands = {0.0}
+    for l in range(L):
+        T = int(cum[l, -1])
+        for c in cum[l]:
+            x = float(Fraction(int(c), T))
+            for _ in range(3):
+                x = np.nextafter(x, 0.0)
+            for _ in range(7):
+                if 0.0 <= x < 1.0:
+                    cands.add(float(x))
+                x = np.nextafter(x, 2.0)
+    best = None
+    for p in sorted(cands):
+        lens = [_length_exact(cum[l], p) for l in range(L)]
+        if sum(lens) <= budget:
+            best = (p, lens)
+        else:
+            break
+    return best
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_search_equals_brute_force(seed):
+    rng = np.random.default_rng(100 + seed)
+    L, N = int(rng.integers(2, 6)), int(rng.integers(3, 24))
+    scores = (rng.random((L, N)) ** rng.integers(1, 5)).astype(np.float32) + np.float32(1e-3)
+    for budget in sorted({L, L + 1, (L * N) // 3, (L * N) // 2, L * N - 1}):
+        if budget < L:
+            continue
+        order, cum, res = oracle.select_sample(scores, budget, tol=0.0, max_iters=4000)
+        assert res.status == oracle.OK
+        p_bf, len_bf = _brute_force_config(cum, budget)
+        assert list(res.len) == len_bf, (budget, res, p_bf)
+        assert res.len.sum() <= budget
+        # with a tolerance the answer is feasible and never better than the optimum
+        _, _, r6 = oracle.select_sample(scores, budget, tol=1e-6)
+        assert r6.len.sum() <= sum(len_bf) <= budget
+        assert r6.iters <= 20
+        assert all(a <= b for a, b in zip(r6.len, len_bf))
+
+
+def test_search_hand_example():
+    A = np.array([11, 3, 2], np.float32) / 16
+    B = np.array([6, 5, 5], np.float32) / 16
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "search_hand_example.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 4
+    for budget, p, la, lb, steps in rows:
+        _, cum, res = oracle.select_sample(np.stack([A, B]), int(budget), tol=0.0, max_iters=4000)
+        assert [int(c) for c in cum[0]] == [11 << 28, 14 << 28, 16 << 28]
+        assert res.p == float(p), (budget, res)
+        assert list(res.len) == [int(la), int(lb)]
+        if int(steps) >= 0:
+            assert res.iters == int(steps)
+
+
+def test_search_invariants():
+    rng = np.random.default_rng(7)
+    L, N = 6, 40
+    scores = np.exp(rng.standard_normal((L, N)) * np.linspace(0.2, 2.5, L)[:, None]).astype(np.float32)
+    prev = None
+    for budget in range(L, L * N + 3, 7):
+        _, cum, res = oracle.select_sample(scores, budget, tol=0.0, max_iters=4000)
+        assert res.len.sum() <= budget
+        assert (res.len >= 1).all() and (res.len <= N).all()
+        if prev is not None:
+            assert (res.len >= prev).all()          # lengths grow with the budget
+        prev = res.len.copy()
+    # full budget keeps everything at p = 1 without a single step
+    _, _, res = oracle.select_sample(scores, L * N)
+    assert res.p == 1.0 and (res.len == N).all() and res.iters == 0
+    # below one row per layer is an error
+    _, _, res = oracle.select_sample(scores, L - 1)
+    assert res.status == oracle.BUDGET_TOO_SMALL
+    # identical layers get identical lengths, floor(budget / L) when nothing ties
+    same = np.tile(scores[3], (L, 1))
+    for budget in (L * 5, L * 5 + 3, L * 17 + 5):
+        _, _, res = oracle.select_sample(same, budget, tol=0.0, max_iters=4000)
+        assert (res.len == budget // L).all(), (budget, res.len)
+    # concentrated layers keep fewer rows than dispersed ones (Sec. 4.3, Fig. 5)
+    _, _, res = oracle.select_sample(scores, L * N // 2, tol=0.0, max_iters=4000)
+    assert res.len[0] > res.len[-1]
+    # tol = 1e-6 stops after exactly 20 halvings unless delta hits zero first
+    _, _, r6 = oracle.select_sample(scores, L * N // 2, tol=1e-6)
+    assert r6.iters <= 20
+    # iteration cap
+    _, _, r3 = oracle.select_sample(scores, L * N // 2, tol=0.0, max_iters=3)
+    assert r3.iters <= 3 and r3.len.sum() <= L * N // 2
+    # one-sided slack: may stop early, never exceeds the budget
+    _, _, rs = oracle.select_sample(scores, L * N // 2, tol=0.0, max_iters=4000, slack=5)
+    assert 0 <= L * N // 2 - rs.len.sum() <= 5
+    assert rs.iters <= res.iters
+
+
+def test_given_lengths_validation():
+    assert oracle.check_lengths([1, 5, 10], 10) == oracle.OK
+    assert oracle.check_lengths([0, 5], 10) == oracle.BAD_LENGTH
+    assert oracle.check_lengths([3, 11], 10) == oracle.BAD_LENGTH
+
+
+# --------------------------------------------------------------------------
+# Compaction (Sec. 3.1, Fig. 2a)
+# --------------------------------------------------------------------------
+def test_compact_keeps_top_ranked_rows_in_position_order():
+    rng = np.random.default_rng(8)
+    H, N, D = 3, 29, 4
+    s = rng.random(N).astype(np.float32)
+    order = oracle.sort_desc(s)
+    src = rng.standard_normal((H, N, D)).astype(np.float32)
+    for ln in (1, 7, N):
+        kept = oracle.retained_positions(order, ln)
+        assert list(kept) == sorted(int(x) for x in order[:ln])
+        # the kept set is exactly the ln largest scores
+        thresh = np.sort(s)[::-1][ln - 1]
+        assert all(s[i] >= thresh for i in kept)
+        rows = oracle.gather_rows(src, kept)
+        np.testing.assert_array_equal(rows, src[:, kept, :].transpose(1, 0, 2))
+
+
+# --------------------------------------------------------------------------
+# Decode attention (Sec. 3.1)
+# --------------------------------------------------------------------------
+def test_decode_matches_library_attention():
+    rng = np.random.default_rng(9)
+    R, H, D = 33, 5, 16
+    q = rng.standard_normal((H, D)).astype(np.float32)
+    kc = rng.standard_normal((R, H, D)).astype(np.float32)
+    vc = rng.standard_normal((R, H, D)).astype(np.float32)
+    scale = 0.31
+    out = oracle.decode_attn(q, kc, vc, scale)
+    qt = torch.from_numpy(q).double()[:, None, :]                     # [H, 1, D]
+    kt = torch.from_numpy(kc).double().permute(1, 0, 2)               # [H, R, D]
+    vt = torch.from_numpy(vc).double().permute(1, 0, 2)
+    ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, scale=scale)[:, 0, :]
+    np.testing.assert_allclose(out, ref.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_decode_special_cases():
+    rng = np.random.default_rng(10)
+    R, H, D = 12, 2, 8
+    q = rng.standard_normal((H, D)).astype(np.float32)
+    kc = rng.standard_normal((R, H, D)).astype(np.float32)
+    vc = rng.standard_normal((R, H, D)).astype(np.float32)
+    # a single row returns its value
+    np.testing.assert_allclose(oracle.decode_attn(q, kc[:1], vc[:1], 1.0), vc[0], rtol=0, atol=0)
+    # constant V comes back unchanged
+    const = np.broadcast_to(np.float32(1.5), vc.shape).copy()
+    np.testing.assert_allclose(oracle.decode_attn(q, kc, const, 1.0), 1.5, rtol=1e-14)
+    # scale 0 gives the mean of the value rows
+    np.testing.assert_allclose(oracle.decode_attn(q, kc, vc, 0.0), vc.mean(axis=0, dtype=np.float64),
+                               rtol=1e-12, atol=1e-15)
+    # the order of cached rows does not matter
+    perm = rng.permutation(R)
+    np.testing.assert_allclose(oracle.decode_attn(q, kc[perm], vc[perm], 0.7),
+                               oracle.decode_attn(q, kc, vc, 0.7), rtol=1e-12, atol=1e-14)
+
+
+def test_full_budget_decode_equals_dense_attention():
+    """p = 1 keeps every prompt row, so decoding over the compacted cache plus
+    the appended row is dense attention over the original K, V."""
+    rng = np.random.default_rng(11)
+    L, H, N, D = 2, 3, 20, 8
+    q = rng.standard_normal((L, H, N, D)).astype(np.float32)
+    k = rng.standard_normal((L, H, N, D)).astype(np.float32)
+    v = rng.standard_normal((L, H, N, D)).astype(np.float32)
+    scores = np.stack([oracle.score_layer(q[l], k[l], 0.35) for l in range(L)])
+    order, cum, res = oracle.select_sample(scores, L * N)
+    assert res.p == 1.0
+    qn, kn, vn = (rng.standard_normal((L, H, D)).astype(np.float32) for _ in range(3))
+    for l in range(L):
+        kept = oracle.retained_positions(order[l], res.len[l])
+        kc = np.concatenate([oracle.gather_rows(k[l], kept), kn[l][None]])
+        vc = np.concatenate([oracle.gather_rows(v[l], kept), vn[l][None]])
+        out = oracle.decode_attn(qn[l], kc, vc, 0.35)
+        kt = torch.from_numpy(np.concatenate([k[l], kn[l][:, None]], axis=1)).double()
+        vt = torch.from_numpy(np.concatenate([v[l], vn[l][:, None]], axis=1)).double()
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(qn[l]).double()[:, None], kt, vt, scale=0.35)[:, 0]
+        np.testing.assert_allclose(out, ref.numpy(), rtol=1e-12, atol=1e-14)
+
+
+# --------------------------------------------------------------------------
+# Lorenz / Gini diagnostic (Sec. 3.2, Fig. 3)
+# --------------------------------------------------------------------------
+def test_gini_closed_forms():
+    N = 50
+    ones = np.ones(N, np.float32)
+    assert abs(oracle.gini(ones, oracle.sort_desc(ones))) < 1e-12
+    onehot = np.zeros(N, np.float32); onehot[3] = 2.0
+    assert abs(oracle.gini(onehot, oracle.sort_desc(onehot)) - (1 - 1 / N)) < 1e-12
+    # linear ramp 1..N: G = (N - 1) / (3 N)  (textbook value for the discrete uniform ramp, trapezoid rule)
+    ramp = np.arange(1, N + 1, dtype=np.float32)
+    g = oracle.gini(ramp, oracle.sort_desc(ramp))
+    x = np.sort(ramp.astype(np.float64))
+    ref = (2 * np.sum(np.arange(1, N + 1) * x) / (N * x.sum())) - (N + 1) / N
+    assert abs(g - ref) < 1e-12
