@@ -1,0 +1,196 @@
+/*
+ * prefixkv.h -- C ABI of the B200 (sm_100a) PrefixKV hot-path library.
+ *
+ * PrefixKV (arXiv 2412.03409) compresses the KV cache of a transformer after
+ * prefilling: every prompt key/value vector gets an importance score from the
+ * causal attention it receives (Sec. 3.2); each layer's vectors are ranked by
+ * that score and their normalised importance is accumulated along the ranking
+ * (the "cumulative priority"); one global information-retention ratio p, found
+ * by binary search, fixes how long a prefix of each layer's ranking is kept so
+ * that the total meets a budget (Sec. 3.3, Eq. 1, Algorithm 1); the kept rows
+ * form per-layer caches of unequal length that decoding then attends over
+ * (Sec. 3.1, Fig. 2a).
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless its comment says "host".  Structs
+ *    passed by pointer (pkv_shape, pkv_cache) live on the host.
+ *  - The caller owns and allocates every buffer, including workspace; the
+ *    library never allocates or frees device memory.
+ *  - Every call only enqueues work on `cuda_stream` (a cudaStream_t passed as
+ *    void*; NULL = default stream) and returns at once.  The int returned is a
+ *    pkv_status from host-side argument validation.  Nothing is synchronised
+ *    and no value is read back to the host.
+ *  - Conditions found on the device are reported per sample in dev_status[B]
+ *    (PKV_DEV_*).  A kernel that finds one still finishes and never touches
+ *    memory outside the caller's buffers; the results of that sample are then
+ *    unspecified.  prefixkv_search / prefixkv_apply_lengths overwrite
+ *    dev_status; later stages only raise it from PKV_DEV_OK.
+ *  - Logical tensor shapes use B (batch), L (layers), H (heads), N (prompt
+ *    tokens), D (head_dim).  "Segment" = one (sample, layer) pair, index b*L+l.
+ *  - Supported: dtype fp32 or bf16; head_dim 64 or 128; N <= 16384;
+ *    H*D*sizeof(element) a multiple of 16 bytes.
+ */
+#ifndef PREFIXKV_H_
+#define PREFIXKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PKV_OK = 0,
+    PKV_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad range, misalignment   */
+    PKV_ERR_UNSUPPORTED = 2, /* dtype / head_dim / prompt_len outside the supported set     */
+    PKV_ERR_WORKSPACE = 3,   /* workspace missing, misaligned (256 B) or too small          */
+    PKV_ERR_CUDA = 4         /* a CUDA runtime call failed (see prefixkv_last_cuda_error)    */
+} pkv_status;
+
+enum { /* per-sample device status word */
+    PKV_DEV_OK = 0,
+    PKV_DEV_BAD_SCORE = 1,        /* NaN, inf or negative importance                   */
+    PKV_DEV_RANGE = 2,            /* fixed-point importance total >= 2^53               */
+    PKV_DEV_BUDGET_TOO_SMALL = 3, /* budget < L (each layer keeps at least one row)     */
+    PKV_DEV_BAD_LENGTH = 4,       /* a given length outside [1, N]                      */
+    PKV_DEV_CAPACITY = 5          /* rows would pass a segment's or the cache's capacity */
+};
+
+typedef enum { PKV_F32 = 0, PKV_BF16 = 1 } pkv_dtype;
+
+typedef struct {
+    int32_t batch, layers, heads, head_dim, prompt_len;
+    int32_t dtype; /* pkv_dtype */
+} pkv_shape;
+
+/* Element strides of a [B, L, H, N, D] tensor; the D stride is 1. */
+typedef struct {
+    int64_t b, l, h, n;
+} pkv_strides;
+
+enum { PKV_WS_SCORE = 0, PKV_WS_SEARCH = 1, PKV_WS_COMPACT = 2, PKV_WS_DECODE = 3 };
+
+/* Bytes of 256-byte-aligned workspace the named call needs for this shape.
+ * Returns 0 for an unknown `which` or an unsupported shape. */
+size_t prefixkv_workspace_bytes(const pkv_shape *shape, int which);
+
+/* Text of the last CUDA error seen by this library on the calling thread (host). */
+const char *prefixkv_last_cuda_error(void);
+
+/*
+ * Importance score, Sec. 3.2:
+ *   a^{h,m,n} = softmax over keys j <= m of scale_l * <q^{h,m}, k^{h,j}>   (causal)
+ *   I[b,l,n]  = (1/H) * sum_h sum_{m >= n} a^{h,m,n}
+ * over all N prompt queries.  The printed formula has no scale; scale_l = 1
+ * reproduces it.
+ *   q, k        [B,L,H,N,D] with the given element strides (D contiguous; every
+ *               stride a multiple of 8 elements for bf16 / 4 for fp32 so that
+ *               rows start on 16 bytes)
+ *   layer_scale [L] fp32
+ *   lse         [B,L,H,N] fp32 or NULL: natural-log sum-exp of each query's scaled
+ *               causal logits, if the caller's prefill attention kept it; when
+ *               NULL the library computes it in a first pass
+ *   scores      [B,L,N] fp32, out
+ * bf16 inputs use tensor cores with fp32 accumulation; fp32 inputs use fp32 FMA.
+ */
+int prefixkv_score(const pkv_shape *shape, const void *q, pkv_strides qs, const void *k,
+                   pkv_strides ks, const float *layer_scale, const float *lse, float *scores,
+                   void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Priority sequence, cumulative priority and the binary search for p
+ * (Sec. 3.2, Sec. 3.3, Eq. 1, Algorithm 1), per sample.
+ *   scores        [B,L,N] fp32, finite and >= 0
+ *   budget_rows   [B] int64: total rows the sample may keep over all layers
+ *                 (the paper's r*L*N); must be >= L
+ *   order         [B,L,N] int32 out: positions by (score descending, position
+ *                 ascending) -- the sorted indices s_l^j
+ *   cum           [B,L,N] uint64 out: inclusive prefix sums along `order` of
+ *                 round-half-even(score * 2^32); cum[..,N-1] is the layer total,
+ *                 so P_l^{j/N} = cum[j-1] / cum[N-1]
+ *   len           [B,L] int32 out: rows kept per layer (R_l * N), each in [1,N]
+ *   p_out         [B] fp64 out: the ratio p the lengths belong to
+ *   iters_out     [B] int32 out: midpoints evaluated
+ * Length rule: p >= 1 keeps N rows; otherwise theta = ceil(p * total) (one fp64
+ * multiply) and len = first 1-based j with cum[j-1] >= theta.
+ * Search: if L*N <= budget, p = 1.  Else bisect [0,1]: stop when the interval is
+ * <= tol wide, after max_iters midpoints, or when fp64 cannot split it; a
+ * midpoint whose total S equals the budget, or misses it from below by at most
+ * slack_rows, is returned at once; S < budget raises the lower end, otherwise
+ * the upper end drops.  On a stop the lower end is returned, so sum(len) never
+ * exceeds the budget.
+ */
+int prefixkv_search(const pkv_shape *shape, const float *scores, const int64_t *budget_rows,
+                    double tol, int32_t max_iters, int64_t slack_rows, int32_t *order,
+                    uint64_t *cum, int32_t *len, double *p_out, int32_t *iters_out,
+                    int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Variant for a configuration fixed in advance (the offline estimate of
+ * Sec. 3.3, last paragraph, or the uniform R_l = r of Sec. 3.2): ranks the rows
+ * as above and takes the lengths from the caller.
+ *   len_in   [L] (per_sample = 0) or [B,L] (per_sample = 1) int32, each in [1,N]
+ *   cum      may be NULL
+ */
+int prefixkv_apply_lengths(const pkv_shape *shape, const float *scores, const int32_t *len_in,
+                           int32_t per_sample, int32_t *order, uint64_t *cum, int32_t *len,
+                           int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Ragged per-layer cache (Fig. 2a).  Rows of segment s occupy
+ * [row_offset[s], row_offset[s] + cap[s]) of k and v; the first len[s] are
+ * valid.  A row is one token's vectors for all heads: [H][D] elements.
+ */
+typedef struct {
+    void *k;                /* [total_cap_rows][H][D], caller-allocated                  */
+    void *v;                /* same                                                      */
+    int64_t *row_offset;    /* [B*L + 1] out: exclusive prefix sum of cap                */
+    int32_t *len;           /* [B*L] out: valid rows; grows by one per decode step       */
+    int32_t *cap;           /* [B*L] out: len after compaction + decode_cap              */
+    int64_t total_cap_rows; /* host: rows allocated; must cover sum(len) + B*L*decode_cap */
+    int32_t decode_cap;     /* host: rows of head-room per segment for decoding          */
+} pkv_cache;
+
+/*
+ * Compression after prefilling (Sec. 3.1; "the top R_l proportion ... retained
+ * in each head", Sec. 3.2): for every segment copy the len top-ranked rows of K
+ * and V, in ascending prompt position, into the packed cache, and fill
+ * row_offset / len / cap.  Segments whose rows would pass total_cap_rows raise
+ * PKV_DEV_CAPACITY and copy nothing.
+ *   k, v    [B,L,H,N,D] with strides, as for prefixkv_score
+ *   order   [B,L,N], len [B,L] from prefixkv_search / prefixkv_apply_lengths
+ *   kept    [B,L,N] int32 out, may be NULL (then workspace holds it): the
+ *           retained positions in ascending order, first len entries valid
+ */
+int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, const void *v,
+                     pkv_strides vs, const int32_t *order, const int32_t *len,
+                     pkv_cache *cache, int32_t *kept, int32_t *dev_status, void *ws,
+                     size_t ws_bytes, void *cuda_stream);
+
+/*
+ * One decode step over the ragged cache (Sec. 3.1: the newest token "interacts
+ * with the cached KV vectors"): for every segment of layers [layer_begin,
+ * layer_end), append k_new / v_new as row len, then
+ *   out[b,l,h,:] = sum_j softmax_j(scale_l * <q[b,l,h], K_j[h]>) * V_j[h]
+ * over all len + 1 rows, and set len += 1.
+ *   q, k_new, v_new, out   [B,L,H,D] contiguous, dtype of the cache
+ * A segment already at capacity raises PKV_DEV_CAPACITY, appends nothing and
+ * writes zeros.  Calls on one cache must not overlap on the GPU.
+ */
+int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, const void *q,
+                         const void *k_new, const void *v_new, const float *layer_scale,
+                         int32_t layer_begin, int32_t layer_end, void *out,
+                         int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Lorenz-curve diagnostic of Sec. 3.2 / Fig. 3: Gini coefficient of each
+ * segment's priority sequence from its cumulative sums (trapezoid rule).
+ *   cum  [B,L,N] from prefixkv_search;  gini [B,L] fp64 out
+ */
+int prefixkv_gini(const pkv_shape *shape, const uint64_t *cum, double *gini, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PREFIXKV_H_ */

@@ -1,0 +1,374 @@
+"""CUDA library vs CPU oracle, stage by stage, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import check_scores, oracle_scores, oracle_select, to_np32
+from paper_2412_03409_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+SCORE_TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-3}     # relative
+DECODE_TOL = {torch.float32: 1e-4, torch.bfloat16: 2e-2}    # max abs
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2412_03409_b200 import api as _api
+    return _api
+
+
+def _session(*a, **kw):
+    from paper_2412_03409_b200.session import Session
+    return Session(*a, **kw)
+
+
+def _u64(t):
+    return t.cpu().numpy().view(np.uint64)
+
+
+# --------------------------------------------------------------------------
+# selection: bit-exact on the oracle's own fp32 scores
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("B,L,N,ratio,tol", [
+    (1, 4, 128, 0.5, 1e-6), (2, 5, 1, 1.0, 1e-6), (3, 7, 33, 0.3, 0.0), (2, 32, 640, 0.2, 1e-6),
+    (1, 40, 2048, 0.2, 1e-6), (2, 3, 1000, 0.1, 0.0), (1, 6, 16384, 0.05, 1e-6), (1, 2, 5000, 0.7, 1e-9),
+])
+def test_selection_bit_exact(api, B, L, N, ratio, tol):
+    scores = np.stack([wl.synthetic_scores(L, N, seed=17 * b + N) for b in range(B)])
+    budgets = [max(L, int(ratio * L * N) + 3 * b) for b in range(B)]
+    iters = 64 if tol > 0 else 2000
+    s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    s.search(torch.tensor(budgets), tol=tol, max_iters=iters, scores=torch.from_numpy(scores).cuda())
+    torch.cuda.synchronize()
+    ref = oracle_select(scores, budgets, tol, iters)
+    assert s.status.cpu().tolist() == [0] * B
+    for b, (order, cum, res) in enumerate(ref):
+        np.testing.assert_array_equal(s.order[b].cpu().numpy(), order)
+        np.testing.assert_array_equal(_u64(s.cum[b]), cum)
+        np.testing.assert_array_equal(s.len[b].cpu().numpy(), res.len)
+        assert s.p[b].item() == res.p
+        assert s.iters[b].item() == res.iters
+        assert int(s.len[b].sum()) <= budgets[b]
+
+
+def test_selection_slack_and_iteration_cap(api):
+    L, N = 8, 300
+    scores = wl.synthetic_scores(L, N, seed=5)[None]
+    for tol, iters, slack in [(0.0, 5, 0), (0.0, 2000, 7), (1e-3, 64, 0), (0.0, 0, 0)]:
+        s = _session(1, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+        s.search(L * N // 3, tol=tol, max_iters=iters, slack_rows=slack,
+                 scores=torch.from_numpy(scores).cuda())
+        _, _, res = oracle_select(scores, [L * N // 3], tol, iters, slack)[0]
+        np.testing.assert_array_equal(s.len[0].cpu().numpy(), res.len)
+        assert s.p[0].item() == res.p and s.iters[0].item() == res.iters
+
+
+def test_selection_degenerate_cases(api):
+    L, N = 4, 64
+    scores = wl.synthetic_scores(L, N, seed=9)
+    batch = np.stack([scores, scores, scores, scores])
+    bad = batch.copy()
+    bad[2, 1, 5] = np.nan
+    bad[3, 0, 0] = -1.0
+    s = _session(4, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    # full budget, minimal budget, NaN, negative
+    s.search(torch.tensor([L * N, L, L * N // 2, L * N // 2]), scores=torch.from_numpy(bad).cuda())
+    st = s.status.cpu().tolist()
+    assert st == [api.DEV_OK, api.DEV_OK, api.DEV_BAD_SCORE, api.DEV_BAD_SCORE]
+    assert s.p[0].item() == 1.0 and bool((s.len[0] == N).all()) and s.iters[0].item() == 0
+    ref = oracle_select(batch[:2], [L * N, L])
+    np.testing.assert_array_equal(s.len[1].cpu().numpy(), ref[1][2].len)
+    assert bool((s.len[1] == 1).all())
+    # below one row per layer
+    s.search(torch.tensor([L - 1, L * 3, L * 3, L * 3]), scores=torch.from_numpy(batch).cuda())
+    assert s.status.cpu().tolist() == [api.DEV_BUDGET_TOO_SMALL, 0, 0, 0]
+    # ties and signed zeros: position decides
+    z = np.zeros((1, 1, 40), np.float32)
+    z[0, 0, ::3] = -0.0
+    z[0, 0, 7] = 2.0
+    z[0, 0, 30] = 2.0
+    s1 = _session(1, 1, 4, 64, 40, torch.float32, np.ones(1), decode_cap=1)
+    s1.search(10, scores=torch.from_numpy(z).cuda())
+    np.testing.assert_array_equal(s1.order[0, 0].cpu().numpy(), oracle.sort_desc(z[0, 0]))
+    # fixed-point range
+    big = np.full((1, 1, 40), 2.0 ** 21, np.float32)
+    s1.search(10, scores=torch.from_numpy(big).cuda())
+    assert s1.status.item() == api.DEV_RANGE
+    _, st_ref = oracle.cumulative(big[0, 0], oracle.sort_desc(big[0, 0]))
+    assert st_ref == oracle.RANGE
+
+
+def test_apply_given_lengths(api):
+    B, L, N = 2, 6, 200
+    scores = np.stack([wl.synthetic_scores(L, N, seed=b) for b in range(B)])
+    s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    dev_scores = torch.from_numpy(scores).cuda()
+    uniform = torch.full((L,), int(0.25 * N), dtype=torch.int32)          # R_l = r for every layer
+    s.apply_lengths(uniform, scores=dev_scores)
+    assert s.status.cpu().tolist() == [0, 0]
+    assert bool((s.len.cpu() == int(0.25 * N)).all())
+    for b in range(B):
+        for l in range(L):
+            np.testing.assert_array_equal(s.order[b, l].cpu().numpy(), oracle.sort_desc(scores[b, l]))
+    per = torch.randint(1, N + 1, (B, L), dtype=torch.int32)
+    s.apply_lengths(per, scores=dev_scores)
+    np.testing.assert_array_equal(s.len.cpu().numpy(), per.numpy())
+    assert oracle.check_lengths(per[0].numpy(), N) == oracle.OK
+    per[1, 2] = N + 1
+    s.apply_lengths(per, scores=dev_scores)
+    assert s.status.cpu().tolist() == [0, api.DEV_BAD_LENGTH]
+    assert oracle.check_lengths(per[1].numpy(), N) == oracle.BAD_LENGTH
+
+
+# --------------------------------------------------------------------------
+# compaction: byte-exact rows, untouched head-room
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,H,D,N", [(torch.float32, 4, 64, 128), (torch.bfloat16, 8, 128, 333),
+                                         (torch.bfloat16, 3, 64, 70), (torch.float32, 2, 128, 50)])
+def test_compact_rows_and_offsets(api, dtype, H, D, N):
+    B, L, cap = 2, 3, 4
+    w = wl.scaled(wl.WORKLOADS["tiny"], B=B, L=L, H=H, D=D, N=N, dtype=dtype, seed=31)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scores = np.stack([wl.synthetic_scores(L, N, seed=b + 50) for b in range(B)])
+    budgets = [L * N // 3, L * N // 2]
+    s = _session(B, L, H, D, N, dtype, np.ones(L), decode_cap=cap, poison=True)
+    s.search(torch.tensor(budgets), scores=torch.from_numpy(scores).cuda())
+    s.compact(k, v)
+    torch.cuda.synchronize()
+    assert s.status.cpu().tolist() == [0, 0]
+    ref = oracle_select(scores, budgets)
+    lens = np.concatenate([r[2].len for r in ref])
+    np.testing.assert_array_equal(s.cache.len.cpu().numpy(), lens)
+    np.testing.assert_array_equal(s.cache.cap.cpu().numpy(), lens + cap)
+    offs = np.concatenate([[0], np.cumsum(lens + cap)])
+    np.testing.assert_array_equal(s.cache.row_offset.cpu().numpy(), offs)
+    ck, cv = to_np32(s.cache.k), to_np32(s.cache.v)
+    for b in range(B):
+        for l in range(L):
+            seg = b * L + l
+            kept = oracle.retained_positions(ref[b][0][l], lens[seg])
+            np.testing.assert_array_equal(s.kept[b, l, :lens[seg]].cpu().numpy(), kept)
+            rk = oracle.gather_rows(to_np32(k[b, l]), kept)
+            rv = oracle.gather_rows(to_np32(v[b, l]), kept)
+            np.testing.assert_array_equal(ck[offs[seg]:offs[seg] + lens[seg]], rk)
+            np.testing.assert_array_equal(cv[offs[seg]:offs[seg] + lens[seg]], rv)
+            assert np.isnan(ck[offs[seg] + lens[seg]:offs[seg + 1]]).all()     # head-room untouched
+    assert np.isnan(ck[offs[-1]:]).all()
+
+
+def test_compact_strided_source_and_capacity(api):
+    B, L, H, D, N = 1, 2, 4, 64, 96
+    w = wl.scaled(wl.WORKLOADS["tiny"], B=B, L=L, H=H, D=D, N=N, dtype=torch.bfloat16, seed=3)
+    q, k, v = wl.make_prompt(w, "cuda")
+    # token-major storage [B, L, N, H, D] viewed as [B, L, H, N, D]
+    k_tm = k.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4)
+    v_tm = v.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4)
+    scores = wl.synthetic_scores(L, N, seed=8)[None]
+    s = _session(B, L, H, D, N, torch.bfloat16, np.ones(L), decode_cap=2)
+    s.search(N, scores=torch.from_numpy(scores).cuda())
+    s.compact(k_tm, v_tm)
+    a_k, a_len = s.cache.k.clone(), s.cache.len.clone()
+    s.compact(k, v)
+    assert torch.equal(a_len, s.cache.len)
+    for seg in range(L):
+        o, n = int(s.cache.row_offset[seg]), int(s.cache.len[seg])
+        assert torch.equal(a_k[o:o + n].view(torch.int16), s.cache.k[o:o + n].view(torch.int16))
+    # a cache too small for the request is reported, not overrun
+    small = _session(B, L, H, D, N, torch.bfloat16, np.ones(L), decode_cap=2, max_budget_rows=10,
+                     poison=True)
+    small.search(N, scores=torch.from_numpy(scores).cuda())
+    small.compact(k, v)
+    assert small.status.item() == api.DEV_CAPACITY
+
+
+# --------------------------------------------------------------------------
+# decode attention
+# --------------------------------------------------------------------------
+def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
+    """Oracle caches per segment, grown step by step; returns the worst |error|."""
+    caches = {}
+    for b in range(w.B):
+        order, _, res = ref_sel[b]
+        for l in range(w.L):
+            kept = oracle.retained_positions(order[l], res.len[l])
+            caches[(b, l)] = [oracle.gather_rows(to_np32(k[b, l]), kept),
+                              oracle.gather_rows(to_np32(v[b, l]), kept)]
+    worst = 0.0
+    for t in range(steps):
+        qd, kn, vn = wl.make_decode_inputs(w, t, "cuda")
+        out = s.decode(qd, kn, vn)
+        torch.cuda.synchronize()
+        got = to_np32(out)
+        for (b, l), (ck, cv) in caches.items():
+            ck = np.concatenate([ck, to_np32(kn[b, l])[None]])
+            cv = np.concatenate([cv, to_np32(vn[b, l])[None]])
+            caches[(b, l)] = [ck, cv]
+            ref = oracle.decode_attn(to_np32(qd[b, l]), ck, cv, float(layer_scale[l]))
+            worst = max(worst, float(np.abs(got[b, l] - ref).max()))
+    return worst
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", {}),
+    ("llava7b_b1", dict(L=3, H=8, N=200, T=5)),
+    ("llava7b_b16", dict(B=3, L=2, H=4, N=97, T=4)),
+    ("tiny", dict(D=128, H=2, T=3)),
+    ("llava7b_b1", dict(L=2, H=5, D=64, N=130, T=3)),
+])
+def test_decode_matches_oracle(api, name, kw):
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 7) for b in range(w.B)])
+    budgets = [w.budget_rows()] * w.B
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T)
+    s.search(torch.tensor(budgets), scores=torch.from_numpy(scores).cuda())
+    s.compact(k, v)
+    ref_sel = oracle_select(scores, budgets)
+    len0 = s.cache.len.clone()
+    worst = _decode_reference(w, s, k, v, ref_sel, w.T, scale)
+    assert worst <= DECODE_TOL[w.dtype], worst
+    assert torch.equal(s.cache.len, len0 + w.T)
+    assert s.status.cpu().tolist() == [0] * w.B
+    # one more step than the head-room allows: reported, length unchanged
+    qd, kn, vn = wl.make_decode_inputs(w, w.T, "cuda")
+    s.decode(qd, kn, vn)
+    assert s.status.cpu().tolist() == [api.DEV_CAPACITY] * w.B
+    assert torch.equal(s.cache.len, len0 + w.T)
+
+
+def test_decode_full_budget_is_dense_attention(api):
+    """p = 1 keeps every row, so the ragged path must equal dense attention over
+    the original K, V plus the appended row (library reference on the host)."""
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=2, H=4, N=150, T=1)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
+    s.search(w.L * w.N, scores=torch.from_numpy(wl.synthetic_scores(w.L, w.N, 1)[None]).cuda())
+    s.compact(k, v)
+    assert s.p.item() == 1.0
+    qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
+    out = s.decode(qd, kn, vn).double().cpu()
+    for l in range(w.L):
+        kk = torch.cat([k[0, l], kn[0, l][:, None]], dim=1).double().cpu()
+        vv = torch.cat([v[0, l], vn[0, l][:, None]], dim=1).double().cpu()
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            qd[0, l].double().cpu()[:, None], kk, vv, scale=float(scale[l]))[:, 0]
+        assert (out[0, l] - ref).abs().max() <= DECODE_TOL[w.dtype]
+
+
+def test_decode_layer_range(api):
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=4, H=4, N=80, T=2)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = torch.from_numpy(wl.synthetic_scores(w.L, w.N, 4)[None]).cuda()
+    a = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    b = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    for s in (a, b):
+        s.search(w.budget_rows(), scores=scores)
+        s.compact(k, v)
+    qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
+    full = a.decode(qd, kn, vn).float().clone()
+    b.out.zero_()
+    for l in range(w.L):                      # a model calls one layer at a time
+        b.decode(qd, kn, vn, layer_begin=l, layer_end=l + 1)
+    assert (full - b.out.float()).abs().max() <= DECODE_TOL[w.dtype]
+    assert torch.equal(a.cache.len, b.cache.len)
+
+
+# --------------------------------------------------------------------------
+# importance score
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", {}),
+    ("tiny", dict(N=1)),
+    ("tiny", dict(N=77, H=3, L=2, D=128)),
+    ("llava7b_b1", dict(L=2, H=4, N=200)),
+    ("llava7b_b1", dict(L=1, H=2, N=640)),
+    ("llava7b_b16", dict(B=2, L=2, H=3, N=129, D=64)),
+    ("longctx_b4", dict(B=1, L=2, H=2, N=1000)),
+])
+def test_score_matches_oracle(api, name, kw):
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
+    got = s.score(q, k).cpu().numpy()
+    ref = oracle_scores(q, k, scale)
+    for (b, l), r in ref.items():
+        check_scores(got[b, l], r, SCORE_TOL[w.dtype])
+        assert abs(got[b, l].astype(np.float64).sum() - w.N) <= 2e-3 * w.N
+    # determinism: a second run gives the same bits
+    again = s.score(q, k).cpu().numpy()
+    np.testing.assert_array_equal(got, again)
+
+
+def test_score_with_caller_lse(api):
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=2, H=4, N=160)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
+    base = s.score(q, k).clone()
+    logits = torch.einsum("blhmd,blhnd->blhmn", q.float(), k.float()) * \
+        torch.from_numpy(scale).cuda().view(1, -1, 1, 1, 1)
+    mask = torch.ones(w.N, w.N, dtype=torch.bool, device="cuda").tril()
+    lse = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1).contiguous()
+    got = s.score(q, k, lse=lse)
+    assert (got - base).abs().max() <= 2e-3 * base.abs().max()
+
+
+# --------------------------------------------------------------------------
+# whole path on the tiny configuration, every output against the oracle
+# --------------------------------------------------------------------------
+def test_whole_path_tiny(api):
+    w = wl.WORKLOADS["tiny"]
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T, poison=True)
+    s.compress(q, k, v, w.budget_rows(), tol=w.tol)
+    torch.cuda.synchronize()
+    ref_scores = oracle_scores(q, k, scale)
+    got_scores = s.scores.cpu().numpy()
+    for (b, l), r in ref_scores.items():
+        check_scores(got_scores[b, l], r, SCORE_TOL[w.dtype])
+    # selection is compared on identical fp32 scores: the library's own
+    ref_sel = oracle_select(got_scores, [w.budget_rows()], w.tol)
+    order, cum, res = ref_sel[0]
+    np.testing.assert_array_equal(s.order[0].cpu().numpy(), order)
+    np.testing.assert_array_equal(s.len[0].cpu().numpy(), res.len)
+    assert s.p.item() == res.p and s.iters.item() == res.iters
+    assert int(s.len.sum()) <= w.budget_rows()
+    # concentrated layers (larger logit scale) keep fewer rows
+    assert s.len[0, 0] > s.len[0, 3]
+    worst = _decode_reference(w, s, k, v, ref_sel, w.T, scale)
+    assert worst <= DECODE_TOL[w.dtype]
+
+
+def test_gini_matches_oracle(api):
+    B, L, N = 2, 5, 300
+    scores = np.stack([wl.synthetic_scores(L, N, seed=b + 70) for b in range(B)])
+    s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    s.search(L * N // 2, scores=torch.from_numpy(scores).cuda())
+    g = torch.empty((B, L), dtype=torch.float64, device="cuda")
+    api.prefixkv_gini(s.shape, s.cum, g)
+    for b in range(B):
+        for l in range(L):
+            ref = oracle.gini(scores[b, l], oracle.sort_desc(scores[b, l]))
+            assert abs(g[b, l].item() - ref) < 1e-6
+
+
+def test_argument_validation_fails_on_the_host(api):
+    s = _session(1, 2, 4, 64, 32, torch.float32, np.ones(2), decode_cap=1)
+    bad = api.make_shape(1, 2, 4, 48, 32, torch.float32)       # unsupported head_dim
+    assert api.lib().prefixkv_search(bad, 1, 1, 0.0, 1, 0, 1, 1, 1, 1, 1, 1, None, 0, None) == \
+        api.PKV_ERR_UNSUPPORTED
+    long = api.make_shape(1, 2, 4, 64, 16385, torch.float32)
+    assert api.prefixkv_workspace_bytes(long, api.WS_SCORE) == 0
+    with pytest.raises(api.PrefixKVError):
+        api.prefixkv_search(s.shape, None, s.budget, 1e-6, 64, 0, s.order, s.cum, s.len, s.p,
+                            s.iters, s.status)
+    with pytest.raises(api.PrefixKVError):                      # workspace too small
+        api.prefixkv_decode_attn(s.shape, s.cache, s.out, s.out, s.out, s.layer_scale, s.out,
+                                 s.status, torch.empty(256, dtype=torch.uint8, device="cuda"))
