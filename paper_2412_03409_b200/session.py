@@ -46,7 +46,7 @@ class Session:
     def search(self, budget_rows, tol=1e-6, max_iters=64, slack_rows=0, scores=None):
         if isinstance(budget_rows, torch.Tensor):
             self.budget.copy_(budget_rows)
-        else:
+        elif budget_rows is not None:          # None: keep the budget already on the device
             self.budget.fill_(int(budget_rows))
         api.prefixkv_search(self.shape, self.scores if scores is None else scores, self.budget, tol,
                             max_iters, slack_rows, self.order, self.cum, self.len, self.p,

@@ -1,6 +1,7 @@
 """Oracle-side drivers shared by the GPU parity tests (host numpy only)."""
 from __future__ import annotations
 
+import multiprocessing
 from concurrent.futures import ProcessPoolExecutor
 
 import numpy as np
@@ -29,7 +30,8 @@ def oracle_scores(q, k, layer_scale, segs=None, workers=8):
         res = [_score_job(j) for j in jobs]
     else:
         oracle.build()
-        with ProcessPoolExecutor(max_workers=workers) as ex:
+        ctx = multiprocessing.get_context("spawn")     # never fork a process that holds a CUDA context
+        with ProcessPoolExecutor(max_workers=workers, mp_context=ctx) as ex:
             res = list(ex.map(_score_job, jobs))
     return dict(zip(segs, res))
 
