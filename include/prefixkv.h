@@ -45,7 +45,8 @@ typedef enum {
     PKV_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, bad range, misalignment   */
     PKV_ERR_UNSUPPORTED = 2, /* dtype / head_dim / prompt_len outside the supported set     */
     PKV_ERR_WORKSPACE = 3,   /* workspace missing, misaligned (256 B) or too small          */
-    PKV_ERR_CUDA = 4         /* a CUDA runtime call failed (see prefixkv_last_cuda_error)    */
+    PKV_ERR_CUDA = 4,        /* a CUDA runtime call failed (see prefixkv_last_cuda_error)    */
+    PKV_ERR_STATIC_LIMIT = 5 /* shape too large for the built-in scratch of a *_static call */
 } pkv_status;
 
 enum { /* per-sample device status word */
@@ -182,6 +183,42 @@ int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, const void *q
                          const void *k_new, const void *v_new, const float *layer_scale,
                          int32_t layer_begin, int32_t layer_end, void *out,
                          int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * The same decode step for callers that have no workspace to give.  (The paper
+ * has no counterpart to this call; it exists for deployment.)
+ *
+ * Who needs it: a serving engine that claimed all free device memory for its
+ * own pool when it started has nothing left for cudaMalloc to return once
+ * requests arrive, and a runtime that must not stall between two tokens cannot
+ * pay for cudaMalloc's implicit device-wide synchronisation.  Such callers
+ * still pass every input and output; only the split-K scratch comes from the
+ * library, as a fixed array of prefixkv_decode_static_limit_bytes() (16 MiB)
+ * that each GPU holds from the moment it loads the library until the process
+ * exits.
+ *
+ *  - The call allocates and frees nothing, on the device or through any
+ *    library.
+ *  - A shape whose scratch need, prefixkv_workspace_bytes(shape,
+ *    PKV_WS_DECODE), is above the limit is refused with PKV_ERR_STATIC_LIMIT
+ *    before anything is launched (prefixkv_last_cuda_error() then holds a
+ *    sentence saying so); use prefixkv_decode_attn for those.
+ *  - The first call on each device looks up the array's device address (that
+ *    device must be current).  Make that first call during start-up, outside
+ *    any stream capture.
+ *  - All calls in the process, on any stream, share the one array per GPU, and
+ *    it keeps whatever the previous call left.  The kernels write every slot
+ *    before reading it, so nothing has to be cleared, but two calls that run
+ *    on the same GPU at the same time overwrite each other's partial results:
+ *    order them on one stream or with events.
+ * Everything else (arguments, results, dev_status) is as for
+ * prefixkv_decode_attn.
+ */
+size_t prefixkv_decode_static_limit_bytes(void);
+int prefixkv_decode_attn_static(const pkv_shape *shape, pkv_cache *cache, const void *q,
+                                const void *k_new, const void *v_new, const float *layer_scale,
+                                int32_t layer_begin, int32_t layer_end, void *out,
+                                int32_t *dev_status, void *cuda_stream);
 
 /*
  * Lorenz-curve diagnostic of Sec. 3.2 / Fig. 3: Gini coefficient of each

@@ -14,14 +14,16 @@ import torch
 
 from . import build as _build
 
-PKV_OK, PKV_ERR_INVALID_ARG, PKV_ERR_UNSUPPORTED, PKV_ERR_WORKSPACE, PKV_ERR_CUDA = range(5)
+(PKV_OK, PKV_ERR_INVALID_ARG, PKV_ERR_UNSUPPORTED, PKV_ERR_WORKSPACE, PKV_ERR_CUDA,
+ PKV_ERR_STATIC_LIMIT) = range(6)
 DEV_OK, DEV_BAD_SCORE, DEV_RANGE, DEV_BUDGET_TOO_SMALL, DEV_BAD_LENGTH, DEV_CAPACITY = range(6)
 WS_SCORE, WS_SEARCH, WS_COMPACT, WS_DECODE = range(4)
 F32, BF16 = 0, 1
 
 EXPORTS = ["prefixkv_workspace_bytes", "prefixkv_last_cuda_error", "prefixkv_score",
            "prefixkv_search", "prefixkv_apply_lengths", "prefixkv_compact",
-           "prefixkv_decode_attn", "prefixkv_gini"]
+           "prefixkv_decode_attn", "prefixkv_gini", "prefixkv_decode_attn_static",
+           "prefixkv_decode_static_limit_bytes"]
 
 
 class Shape(ctypes.Structure):
@@ -66,8 +68,12 @@ def _load():
     lib.prefixkv_decode_attn.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp, i32, i32,
                                          vp, vp, vp, sz, vp]
     lib.prefixkv_gini.argtypes = [sp, vp, vp, vp]
-    for name in EXPORTS[2:]:
+    lib.prefixkv_decode_attn_static.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp,
+                                                i32, i32, vp, vp, vp]
+    for name in EXPORTS[2:-1]:
         getattr(lib, name).restype = ctypes.c_int
+    lib.prefixkv_decode_static_limit_bytes.restype = ctypes.c_size_t
+    lib.prefixkv_decode_static_limit_bytes.argtypes = []
     return lib
 
 
@@ -80,9 +86,9 @@ def lib():
 
 def _check(rc, what):
     if rc != PKV_OK:
-        names = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CUDA"]
-        extra = _lib.prefixkv_last_cuda_error().decode() if rc == PKV_ERR_CUDA else ""
-        raise PrefixKVError("%s failed: PKV_ERR_%s %s" % (what, names[rc] if rc < 5 else rc, extra))
+        names = ["OK", "INVALID_ARG", "UNSUPPORTED", "WORKSPACE", "CUDA", "STATIC_LIMIT"]
+        extra = _lib.prefixkv_last_cuda_error().decode() if rc >= PKV_ERR_CUDA else ""
+        raise PrefixKVError("%s failed: PKV_ERR_%s %s" % (what, names[rc] if rc < 6 else rc, extra))
 
 
 def _ptr(t):
@@ -192,3 +198,21 @@ def prefixkv_decode_attn(shape, cache: Cache, q, k_new, v_new, layer_scale, out,
 
 def prefixkv_gini(shape, cum, gini):
     _check(_lib.prefixkv_gini(ctypes.byref(shape), _ptr(cum), _ptr(gini), _stream()), "prefixkv_gini")
+
+
+def prefixkv_decode_static_limit_bytes() -> int:
+    return int(_lib.prefixkv_decode_static_limit_bytes())
+
+
+def prefixkv_decode_attn_static(shape, cache: Cache, q, k_new, v_new, layer_scale, out, dev_status,
+                                layer_begin=0, layer_end=None):
+    """Decode step that takes no workspace: for callers that cannot allocate device
+    memory by the time they decode (all of it already sits in their own pool, or an
+    allocation's device-wide synchronisation is not acceptable between tokens).  The
+    split-K scratch is a fixed 16 MiB array inside the library; larger shapes raise.
+    Calls share that array, so do not let two of them overlap on one GPU."""
+    le = shape.layers if layer_end is None else layer_end
+    _check(_lib.prefixkv_decode_attn_static(ctypes.byref(shape), ctypes.byref(cache.c), _ptr(q),
+                                            _ptr(k_new), _ptr(v_new), _ptr(layer_scale),
+                                            int(layer_begin), int(le), _ptr(out), _ptr(dev_status),
+                                            _stream()), "prefixkv_decode_attn_static")

@@ -14,6 +14,8 @@ void set_cuda_error(cudaError_t e, const char *where)
     snprintf(g_err, sizeof(g_err), "%s: %s", where, cudaGetErrorString(e));
 }
 
+void set_error_text(const char *text) { snprintf(g_err, sizeof(g_err), "%s", text); }
+
 int check_launch(const char *where)
 {
     cudaError_t e = cudaGetLastError();

@@ -13,6 +13,7 @@ constexpr size_t kWsAlign = 256;
 
 // Host-side record of the last CUDA error (thread local).
 void set_cuda_error(cudaError_t e, const char *where);
+void set_error_text(const char *text);
 int check_launch(const char *where);
 // Raises a kernel's dynamic shared-memory limit once per device.
 int ensure_dynamic_smem(const void *func, int bytes, bool *done_per_device);

@@ -223,3 +223,79 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
     }
 #undef PKV_DEC
 }
+
+// ---------------------------------------------------------------------------
+// Decode step for callers that cannot hand over workspace.
+//
+// Some callers of this library are not able to obtain device memory when they
+// reach the decode loop: a serving engine that gave every free byte to its own
+// pool at start-up has nothing left for cudaMalloc to return, and a runtime that
+// must never stall cannot afford cudaMalloc's implicit device-wide
+// synchronisation between two tokens.  For them the split-K partials live in a
+// fixed device array that is part of the library image: every GPU that loads
+// the library carries kStaticScratchBytes for it until the process exits.
+//
+// In host code the array's name only stands for the symbol; it is not a device
+// address.  The real address is looked up once per device with
+// cudaGetSymbolAddress (while that device is current) and handed to the same
+// kernels the workspace entry point launches.
+// ---------------------------------------------------------------------------
+#include <mutex>
+
+namespace pkv {
+
+constexpr size_t kStaticScratchBytes = 16u << 20;  // 16 MiB per GPU
+static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
+
+static int static_scratch_address(void **out)
+{
+    static std::mutex mu;
+    static void *addr[64] = {};
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "cudaGetDevice");
+        return PKV_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= 64) {
+        set_cuda_error(cudaErrorInvalidDevice, "static scratch: device index above 63");
+        return PKV_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_decode_scratch);
+        if (e != cudaSuccess || !p) {
+            set_cuda_error(e, "cudaGetSymbolAddress(decode scratch)");
+            return PKV_ERR_CUDA;
+        }
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return PKV_OK;
+}
+
+}  // namespace pkv
+
+extern "C" size_t prefixkv_decode_static_limit_bytes(void) { return pkv::kStaticScratchBytes; }
+
+extern "C" int prefixkv_decode_attn_static(const pkv_shape *shape, pkv_cache *cache, const void *q,
+                                           const void *k_new, const void *v_new,
+                                           const float *layer_scale, int32_t layer_begin,
+                                           int32_t layer_end, void *out, int32_t *dev_status,
+                                           void *cuda_stream)
+{
+    if (!shape_ok(shape)) return PKV_ERR_INVALID_ARG;
+    if (!shape_supported(shape)) return PKV_ERR_UNSUPPORTED;
+    const size_t need = decode_ws_bytes(shape);
+    if (need > kStaticScratchBytes) {
+        set_error_text("prefixkv_decode_attn_static: this shape needs more scratch than the "
+                       "built-in 16 MiB array; use prefixkv_decode_attn with caller workspace");
+        return PKV_ERR_STATIC_LIMIT;
+    }
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != PKV_OK) return rc;
+    return prefixkv_decode_attn(shape, cache, q, k_new, v_new, layer_scale, layer_begin, layer_end,
+                                out, dev_status, scratch, kStaticScratchBytes, cuda_stream);
+}
