@@ -55,7 +55,8 @@ enum { /* per-sample device status word */
     PKV_DEV_RANGE = 2,            /* fixed-point importance total >= 2^53               */
     PKV_DEV_BUDGET_TOO_SMALL = 3, /* budget < L (each layer keeps at least one row)     */
     PKV_DEV_BAD_LENGTH = 4,       /* a given length outside [1, N]                      */
-    PKV_DEV_CAPACITY = 5          /* rows would pass a segment's or the cache's capacity */
+    PKV_DEV_CAPACITY = 5,         /* rows would pass a segment's or the cache's capacity */
+    PKV_DEV_TIMEOUT = 6           /* a bounded wait inside a kernel ran out (reported on sample 0) */
 };
 
 typedef enum { PKV_F32 = 0, PKV_BF16 = 1 } pkv_dtype;
@@ -149,6 +150,9 @@ typedef struct {
     int64_t *row_offset;    /* [B*L + 1] out: exclusive prefix sum of cap                */
     int32_t *len;           /* [B*L] out: valid rows; grows by one per decode step       */
     int32_t *cap;           /* [B*L] out: len after compaction + decode_cap              */
+    int32_t *arrive;        /* [B*L + 1]: arrival counters of the decode kernel; zeroed by
+                               prefixkv_compact, zero again after every decode call.  May be
+                               NULL: decoding then takes a slower two-kernel path.          */
     int64_t total_cap_rows; /* host: rows allocated; must cover sum(len) + B*L*decode_cap */
     int32_t decode_cap;     /* host: rows of head-room per segment for decoding          */
 } pkv_cache;

@@ -160,13 +160,19 @@ static int pick_splits(int nseg_active)
     return s < 1 ? 1 : (s > 64 ? 64 : s);
 }
 
+size_t decode_stream_ws_bytes(const pkv_shape *s);
+int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const void *kn,
+                         const void *vn, const float *scale, int lb, int le, void *out,
+                         int32_t *dev_status, void *ws, cudaStream_t st);
+
 size_t decode_ws_bytes(const pkv_shape *s)
 {
-    // splits * active segments never exceeds 148 * 4 + B * L partial slots.
+    // Two-kernel path: splits * active segments never exceeds 148 * 4 + B * L partial slots.
     size_t nseg = (size_t)s->batch * s->layers;
     size_t slots = 148 * 4 + nseg;
     size_t per = (size_t)s->heads * (s->head_dim + 2) * sizeof(float);
-    return round_up(slots * per, kWsAlign);
+    size_t two = round_up(slots * per, kWsAlign), one = decode_stream_ws_bytes(s);
+    return two > one ? two : one;
 }
 
 template <typename T, int D>
@@ -211,6 +217,11 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
     if ((size_t)shape->batch * (layer_end - layer_begin) > 65535) return PKV_ERR_UNSUPPORTED;
     if (!ws || !aligned(ws, kWsAlign) || ws_bytes < decode_ws_bytes(shape)) return PKV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    {
+        int rc = launch_decode_stream(shape, cache, q, k_new, v_new, layer_scale, layer_begin,
+                                      layer_end, out, dev_status, ws, st);
+        if (rc >= 0) return rc;  // -1: shape outside the streaming kernel, use the two-kernel path
+    }
 #define PKV_DEC(T, D)                                                                              \
     return launch_decode<T, D>(shape, cache, q, k_new, v_new, layer_scale, layer_begin, layer_end, \
                                out, dev_status, ws, st)
