@@ -150,9 +150,6 @@ typedef struct {
     int64_t *row_offset;    /* [B*L + 1] out: exclusive prefix sum of cap                */
     int32_t *len;           /* [B*L] out: valid rows; grows by one per decode step       */
     int32_t *cap;           /* [B*L] out: len after compaction + decode_cap              */
-    int32_t *arrive;        /* [B*L + 1]: arrival counters of the decode kernel; zeroed by
-                               prefixkv_compact, zero again after every decode call.  May be
-                               NULL: decoding then takes a slower two-kernel path.          */
     int64_t total_cap_rows; /* host: rows allocated; must cover sum(len) + B*L*decode_cap */
     int32_t decode_cap;     /* host: rows of head-room per segment for decoding          */
 } pkv_cache;
@@ -181,7 +178,8 @@ int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, cons
  * over all len + 1 rows, and set len += 1.
  *   q, k_new, v_new, out   [B,L,H,D] contiguous, dtype of the cache
  * A segment already at capacity raises PKV_DEV_CAPACITY, appends nothing and
- * writes zeros.  Calls on one cache must not overlap on the GPU.
+ * writes zeros.  Calls on one cache, or sharing one workspace, must not overlap on
+ * the GPU.
  */
 int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, const void *q,
                          const void *k_new, const void *v_new, const float *layer_scale,

@@ -40,7 +40,7 @@ class Strides(ctypes.Structure):
 
 class CacheStruct(ctypes.Structure):
     _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("row_offset", ctypes.c_void_p),
-                ("len", ctypes.c_void_p), ("cap", ctypes.c_void_p), ("arrive", ctypes.c_void_p),
+                ("len", ctypes.c_void_p), ("cap", ctypes.c_void_p),
                 ("total_cap_rows", ctypes.c_int64), ("decode_cap", ctypes.c_int32)]
 
 
@@ -155,20 +155,17 @@ class Cache:
     row_offset: torch.Tensor
     len: torch.Tensor
     cap: torch.Tensor
-    arrive: torch.Tensor
     total_cap_rows: int
     decode_cap: int
     c: CacheStruct = None
 
     def __post_init__(self):
         self.c = CacheStruct(self.k.data_ptr(), self.v.data_ptr(), self.row_offset.data_ptr(),
-                             self.len.data_ptr(), self.cap.data_ptr(),
-                             self.arrive.data_ptr() if self.arrive is not None else None,
-                             self.total_cap_rows, self.decode_cap)
+                             self.len.data_ptr(), self.cap.data_ptr(), self.total_cap_rows,
+                             self.decode_cap)
 
 
-def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=None,
-                with_arrive=True) -> Cache:
+def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=None) -> Cache:
     """total_rows: host-known upper bound on the retained rows of all samples."""
     nseg = shape.batch * shape.layers
     dt = torch.float32 if shape.dtype == F32 else torch.bfloat16
@@ -180,9 +177,7 @@ def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=Non
     return Cache(mk(cap_rows, shape.heads, shape.head_dim), mk(cap_rows, shape.heads, shape.head_dim),
                  torch.zeros(nseg + 1, dtype=torch.int64, device=device),
                  torch.zeros(nseg, dtype=torch.int32, device=device),
-                 torch.zeros(nseg, dtype=torch.int32, device=device),
-                 torch.zeros(nseg + 1, dtype=torch.int32, device=device) if with_arrive else None,
-                 cap_rows, int(decode_cap))
+                 torch.zeros(nseg, dtype=torch.int32, device=device), cap_rows, int(decode_cap))
 
 
 def prefixkv_compact(shape, k, v, order, length, cache: Cache, dev_status, ws, kept=None):

@@ -13,8 +13,7 @@ __global__ void __launch_bounds__(1024)
 compact_plan_kernel(const int32_t *__restrict__ order, const int32_t *__restrict__ len_in, int nseg,
                     int L, int N, int decode_cap, int64_t total_cap_rows,
                     int64_t *__restrict__ row_offset, int32_t *__restrict__ len_out,
-                    int32_t *__restrict__ cap_out, int32_t *__restrict__ arrive,
-                    int32_t *__restrict__ kept, int32_t *dev_status)
+                    int32_t *__restrict__ cap_out, int32_t *__restrict__ kept, int32_t *dev_status)
 {
     __shared__ uint32_t bitmap[kMaxPromptLen / 32];
     __shared__ int64_t red[32];
@@ -52,10 +51,6 @@ compact_plan_kernel(const int32_t *__restrict__ order, const int32_t *__restrict
         if (seg == nseg - 1) row_offset[nseg] = off + cap;
         len_out[seg] = fits ? n : 0;
         cap_out[seg] = fits ? cap : 0;
-        if (arrive) {
-            arrive[seg] = 0;
-            if (seg == nseg - 1) arrive[nseg] = 0;
-        }
     }
     if (!fits) n = 0;
 
@@ -168,8 +163,7 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     compact_plan_kernel<<<nseg, 1024, 0, stream>>>(order, len, nseg, L, N, cache->decode_cap,
                                                    cache->total_cap_rows, cache->row_offset,
-                                                   cache->len, cache->cap, cache->arrive, kept,
-                                                   dev_status);
+                                                   cache->len, cache->cap, kept, dev_status);
     int rc = check_launch("compact_plan_kernel");
     if (rc != PKV_OK) return rc;
 

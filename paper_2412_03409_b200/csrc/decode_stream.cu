@@ -1,24 +1,27 @@
 // Streaming decode attention over the ragged cache (Sec. 3.1, Fig. 2a), the
 // bandwidth-bound form of the decode step.
 //
-// Work is cut into units of up to four consecutive cache rows of one segment and
-// the flat unit list is divided evenly over one persistent CTA per SM, so ragged
-// per-layer lengths cost no imbalance.  A producer thread streams each unit's K
-// rows and V rows (contiguous in the token-major cache) into a shared-memory ring
-// with bulk asynchronous copies that complete on mbarriers; consumer warps own
-// heads, keep q, the running softmax state and the output accumulator in
-// registers, and read the ring with conflict-free 16-byte loads.  A CTA that
-// covers only part of a segment leaves an un-normalised partial in scratch; the
-// last CTA to arrive at the segment (a counter, no waiting) merges them.  The
-// last CTA of the grid bumps the lengths, after every CTA has read them.
+// Work is cut into units of up to UR consecutive rows of one segment (the row
+// being appended counts as the segment's last row) and the flat unit list is
+// divided evenly over one persistent CTA per SM, so ragged per-layer lengths cost
+// no imbalance.  One producer thread moves everything the CTA reads -- q, each
+// unit's K rows and V rows (contiguous in the token-major cache) and the new
+// k/v row -- into shared memory with bulk asynchronous copies that complete on
+// mbarriers; no other thread loads from global memory while the stream runs, so
+// nothing queues behind the bulk traffic.  Consumer warps own heads, keep q, the
+// running softmax state and the output accumulator in registers, and read the
+// ring with conflict-free 16-byte loads.  A CTA that covers a whole segment
+// writes its output directly; one that covers part of it leaves an
+// un-normalised partial in scratch.  A small second kernel, launched as a
+// programmatic dependent so that its launch overlaps the stream, merges the
+// partials of split segments in parallel over all SMs and bumps the lengths.
 #include <cstdlib>
 
 #include "common.cuh"
 
 namespace pkv {
 
-constexpr int kUnitRows = 4;
-constexpr int kMaxActive = 2048;
+constexpr int kMaxActive = 1024;
 constexpr int kMaxStages = 8;
 constexpr int kDynSmemMax = 226 * 1024;  // 227 KiB per CTA less the kernel's static variables
 constexpr uint32_t kSpinLimit = 1u << 22;
@@ -30,12 +33,13 @@ struct DecodeArgs {
     const int64_t *row_offset;
     int32_t *len;
     const int32_t *cap;
-    int32_t *arrive;  // [B*L + 1], zero between calls
     const float *layer_scale;
-    float *scratch;
+    float *scratch;   // partial slots
+    int *plan;        // [4 + (nact + 1) + nact]: U, G, units per CTA, remainder; unit prefix; rows
     int32_t *dev_status;
     int L, H, layer_begin, nl, nact, nseg_total, nstages, nwarps;
     uint32_t row_bytes;
+    int64_t total_cap_rows;
 };
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p)
@@ -120,69 +124,105 @@ template <> struct Vec<__nv_bfloat16> {
     }
 };
 
-// Owner CTA of unit u when U units are spread over G CTAs as [floor(cU/G), floor((c+1)U/G)).
-__device__ __forceinline__ int unit_owner(int u, int G, int U)
+// U units over G CTAs (G <= U): the first U % G CTAs take U / G + 1 units, the rest U / G.
+__device__ __forceinline__ int first_unit(int c, int q, int rem) { return c * q + min(c, rem); }
+__device__ __forceinline__ int unit_owner(int u, int q, int rem)
 {
-    return (int)((((int64_t)u + 1) * G - 1) / U);
+    const int big = rem * (q + 1);
+    return u < big ? u / (q + 1) : rem + (u - big) / q;
 }
 
+// Wait for a barrier phase; `dead` latches once a bounded wait has run out anywhere in
+// the CTA, after which nothing waits any more (the results are then unspecified).
+__device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag)
+{
+    if (dead || mbar_try_wait(bar, parity)) return;
+    if (*(volatile int *)abort_flag || !mbar_wait(bar, parity)) {
+        dead = true;
+        atomicExch(abort_flag, 1);
+    }
+}
+
+struct Ring {
+    int slot, nstages;
+    uint32_t phase;
+    __device__ __forceinline__ void advance()
+    {
+        if (++slot == nstages) {
+            slot = 0;
+            phase ^= 1u;
+        }
+    }
+};
+
 // LPR lanes share one (row, head): lane c of a group holds 16-byte vectors c, c + LPR, ...
-// HPW heads per consumer warp.  Block = nwarps consumer warps + 1 producer warp.
-template <typename T, int D, int LPR, int HPW, int MAXT>
+// HPW heads per consumer warp, UR rows per unit.  Block = nwarps consumer warps + 1 producer warp.
+template <typename T, int D, int LPR, int HPW, int UR, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs a)
 {
     constexpr int VE = Vec<T>::VE;
     constexpr int NV = D / VE / LPR;  // vectors per lane
     constexpr int EPL = NV * VE;      // elements per lane
     constexpr int GPW = 32 / LPR;     // row groups per warp
-    static_assert(NV >= 1, "too many lanes per row");
+    constexpr int RPG = UR / GPW;     // rows per group per unit
     constexpr int kSlotStride = D + 4;  // acc[D], max, sum; padded so every head starts on 16 bytes
+    static_assert(NV >= 1 && RPG >= 1, "bad lane mapping");
 
     extern __shared__ __align__(128) unsigned char smem[];
-    const uint32_t slot_bytes = kUnitRows * a.row_bytes;
+    const uint32_t rb = a.row_bytes;
+    const uint32_t slot_bytes = UR * rb;
     unsigned char *ring = smem;
-    uint64_t *full = reinterpret_cast<uint64_t *>(smem + (size_t)a.nstages * slot_bytes);
+    unsigned char *qbuf = ring + (size_t)a.nstages * slot_bytes;  // [2][rb]
+    uint64_t *full = reinterpret_cast<uint64_t *>(qbuf + 2 * (size_t)rb);
     uint64_t *empty = full + kMaxStages;
-    int *P = reinterpret_cast<int *>(empty + kMaxStages);  // [nact + 1] unit prefix
-    int *nlen = P + a.nact + 1;                            // [nact] rows, or -1 when not active
-    __shared__ int s_flag, s_abort;
+    uint64_t *qfull = empty + kMaxStages;  // [2]
+    uint64_t *qempty = qfull + 2;          // [2]
+    int64_t *seg_off = reinterpret_cast<int64_t *>(qempty + 2);  // [nact] first row of the segment
+    int *P = reinterpret_cast<int *>(seg_off + a.nact);          // [nact + 1] unit prefix
+    int *seg_n = P + a.nact + 1;                                 // [nact] rows, or -1 when not active
+    __shared__ int s_abort;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int NW = a.nwarps;
     const int H = a.H;
 
-    // ---- plan: units per active segment, exclusive scan (warp 0) -------------------------
+    // ---- plan: rows, first row and unit count of every active segment ---------------------
     if (tid == 0) {
         s_abort = 0;
         for (int i = 0; i < a.nstages; ++i) {
             mbar_init(full + i, 1);
             mbar_init(empty + i, NW);
         }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(qfull + i, 1);
+            mbar_init(qempty + i, NW);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        P[0] = 0;
     }
+    for (int si = tid; si < a.nact; si += blockDim.x) {
+        const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+        const int ln = a.len[seg], cp = a.cap[seg];
+        const int64_t off = a.row_offset[seg];
+        const bool ok = ln >= 1 && ln < cp && off >= 0 && off + cp <= a.total_cap_rows;
+        seg_n[si] = ok ? ln : -1;
+        seg_off[si] = off;
+        P[si + 1] = ok ? (ln + UR) / UR : 0;  // ceil((ln + 1) / UR): the appended row is the last row
+    }
+    __syncthreads();
     if (warp == 0) {
         int run = 0;
         for (int base = 0; base < a.nact; base += 32) {
-            int si = base + lane, units = 0, n = -1;
-            if (si < a.nact) {
-                int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-                int ln = a.len[seg], cp = a.cap[seg];
-                if (ln >= 1 && ln < cp) {
-                    n = ln;
-                    units = (ln + kUnitRows - 1) / kUnitRows;
-                }
-                nlen[si] = n;
-            }
-            int incl = units;
+            const int i = base + lane;
+            int incl = i < a.nact ? P[i + 1] : 0;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 int up = __shfl_up_sync(0xffffffffu, incl, o);
                 if (lane >= o) incl += up;
             }
-            if (si < a.nact) P[si] = run + incl - units;
+            if (i < a.nact) P[i + 1] = run + incl;
             run += __shfl_sync(0xffffffffu, incl, 31);
         }
-        if (lane == 0) P[a.nact] = run;
     }
     __syncthreads();
     const int U = P[a.nact];
@@ -191,90 +231,120 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 
     // segments that cannot take another row: report, write zeros
     for (int si = cta; si < a.nact; si += gridDim.x) {
-        if (nlen[si] >= 0) continue;
+        if (seg_n[si] >= 0) continue;
         const int b = si / a.nl, seg = b * a.L + a.layer_begin + si % a.nl;
         if (tid == 0) raise_status(a.dev_status, b, PKV_DEV_CAPACITY);
         T *o = reinterpret_cast<T *>(a.out) + (size_t)seg * H * D;
         for (int e = tid; e < H * D; e += blockDim.x) o[e] = from_float<T>(0.f);
     }
 
-    int u0 = 0, u1 = 0;
+    int u0 = 0, u1 = 0, si0 = 0;
+    const int upc = G > 0 ? U / G : 0, rem = G > 0 ? U - upc * G : 0;
+    // The merge kernel may be scheduled from here on; it still waits for this grid to finish.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (cta == 0) {  // the plan, for the merge kernel
+        if (tid == 0) {
+            a.plan[0] = U; a.plan[1] = G; a.plan[2] = upc; a.plan[3] = rem;
+        }
+        for (int i = tid; i <= a.nact; i += blockDim.x) a.plan[4 + i] = P[i];
+        for (int i = tid; i < a.nact; i += blockDim.x) a.plan[5 + a.nact + i] = seg_n[i];
+    }
     if (cta < G) {
-        u0 = (int)((int64_t)cta * U / G);
-        u1 = (int)((int64_t)(cta + 1) * U / G);
+        u0 = first_unit(cta, upc, rem);
+        u1 = first_unit(cta + 1, upc, rem);
+        int lo = 0, hi = a.nact;  // last segment whose first unit is <= u0
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (P[mid] <= u0) lo = mid; else hi = mid;
+        }
+        si0 = lo;
     }
 
     if (warp == NW) {
-        // ---- producer ---------------------------------------------------------------------
+        // ---- producer: the only thread that reads global memory while the stream runs --------
         if (lane == 0 && u0 < u1) {
-            int si = 0, it = 0;
-            // binary search for the segment of u0
-            {
-                int lo = 0, hi = a.nact;
-                while (hi - lo > 1) {
-                    int mid = (lo + hi) >> 1;
-                    if (P[mid] <= u0) lo = mid; else hi = mid;
+            Ring r{0, a.nstages, 0u};
+            int qi = 0;
+            uint32_t qph = 0;
+            int si = si0, issued = 0;
+            bool dead = false, piece_start = true;
+            int n = 0, r0 = 0, seg = 0;
+            int64_t off = 0;
+            for (int u = u0; u < u1 && !dead; ++u) {
+                if (u >= P[si + 1]) {
+                    do ++si; while (u >= P[si + 1]);
+                    piece_start = true;
                 }
-                si = lo;
-            }
-            bool ok = true;
-            for (int u = u0; u < u1 && ok; ++u) {
-                while (u >= P[si + 1]) ++si;
-                const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-                const int r0 = (u - P[si]) * kUnitRows;
-                const int cnt = min(kUnitRows, nlen[si] - r0);
-                const uint32_t bytes = (uint32_t)cnt * a.row_bytes;
-                const size_t src_off = (size_t)(a.row_offset[seg] + r0) * a.row_bytes;
+                if (piece_start) {
+                    piece_start = false;
+                    seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+                    n = seg_n[si];
+                    off = seg_off[si];
+                    r0 = (u - P[si]) * UR;
+                    wait_phase(qempty + qi, qph ^ 1u, dead, &s_abort);
+                    if (dead) break;
+                    mbar_expect_tx(qfull + qi, rb);
+                    bulk_load(qbuf + (size_t)qi * rb, reinterpret_cast<const unsigned char *>(a.q) + (size_t)seg * rb,
+                              rb, qfull + qi);
+                    qi ^= 1;
+                    if (qi == 0) qph ^= 1u;
+                }
+                const int from_cache = min(UR, max(n - r0, 0));
+                const bool has_new = r0 + UR > n;  // this unit ends the segment
+                const uint32_t bytes = (uint32_t)(from_cache + (has_new ? 1 : 0)) * rb;
 #pragma unroll
                 for (int kv = 0; kv < 2; ++kv) {
-                    const int slot = it % a.nstages;
-                    const uint32_t ph = (uint32_t)(it / a.nstages) & 1u;
-                    if (!mbar_wait(empty + slot, ph ^ 1u) || *(volatile int *)&s_abort) {
-                        atomicExch(&s_abort, 1);
-                        ok = false;
-                        break;
-                    }
-                    mbar_expect_tx(full + slot, bytes);
-                    const unsigned char *src =
-                        reinterpret_cast<const unsigned char *>(kv ? a.cv : a.ck) + src_off;
-                    bulk_load(ring + (size_t)slot * slot_bytes, src, bytes, full + slot);
-                    ++it;
+                    wait_phase(empty + r.slot, r.phase ^ 1u, dead, &s_abort);
+                    if (dead) break;
+                    unsigned char *dst = ring + (size_t)r.slot * slot_bytes;
+                    mbar_expect_tx(full + r.slot, bytes);
+                    if (from_cache > 0)
+                        bulk_load(dst, reinterpret_cast<const unsigned char *>(kv ? a.cv : a.ck) + (size_t)(off + r0) * rb,
+                                  (uint32_t)from_cache * rb, full + r.slot);
+                    if (has_new)
+                        bulk_load(dst + (size_t)from_cache * rb,
+                                  reinterpret_cast<const unsigned char *>(kv ? a.v_new : a.k_new) + (size_t)seg * rb, rb,
+                                  full + r.slot);
+                    r.advance();
+                    ++issued;
                 }
+                r0 += UR;
             }
-            if (!ok) {
-                // let copies already issued land before the CTA can exit
-                for (int j = 0; j < it; ++j)
-                    if (it - j <= a.nstages) mbar_wait(full + j % a.nstages, (uint32_t)(j / a.nstages) & 1u);
+            if (dead) {
+                // let copies already issued land before the CTA can exit (bounded)
+                for (int i = 0; i < a.nstages && i < issued; ++i) mbar_wait(full + i, 0u);
             }
         }
     } else if (u0 < u1) {
         // ---- consumers --------------------------------------------------------------------
         const int g = lane / LPR, c = lane % LPR;
-        const int h0 = warp * HPW;
-        float qf[HPW][EPL], acc[HPW][EPL], m[HPW], l[HPW], s[HPW][kUnitRows / GPW];
-        int si = 0, it = 0;
-        {
-            int lo = 0, hi = a.nact;
-            while (hi - lo > 1) {
-                int mid = (lo + hi) >> 1;
-                if (P[mid] <= u0) lo = mid; else hi = mid;
-            }
-            si = lo;
-        }
-        bool fresh = true;  // state must be reset and q loaded for segment si
-        bool timed_out = false;
+        const int h0 = warp * HPW;  // H is a multiple of HPW (checked by the launcher)
+        const uint32_t lane_off = (uint32_t)h0 * D * sizeof(T) + c * 16;
+        float qf[HPW][EPL], acc[HPW][EPL], m[HPW], l[HPW];
+        Ring r{0, a.nstages, 0u};
+        int qi = 0;
+        uint32_t qph = 0;
+        int si = si0;
+        bool dead = false, piece_start = true;
+        int n = 0, r0 = 0, seg = 0, seg_last_u = 0;
+        int64_t off = 0;
+        size_t seg_vec = 0;
         for (int u = u0; u < u1; ++u) {
-            if (u >= P[si + 1]) {
-                while (u >= P[si + 1]) ++si;
-                fresh = true;
+            if (u > seg_last_u && !piece_start) {
+                piece_start = true;
             }
-            const int b = si / a.nl, lyr = a.layer_begin + si % a.nl;
-            const int seg = b * a.L + lyr;
-            const int n = nlen[si];
-            const size_t seg_vec = (size_t)seg * H * D;
-            if (fresh) {
-                fresh = false;
-                const float sc = a.layer_scale[lyr] * kLog2eD;
+            if (piece_start) {
+                piece_start = false;
+                while (u >= P[si + 1]) ++si;
+                seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+                n = seg_n[si];
+                off = seg_off[si];
+                r0 = (u - P[si]) * UR;
+                seg_last_u = P[si + 1] - 1;
+                seg_vec = (size_t)seg * H * D;
+                const float sc = a.layer_scale[a.layer_begin + si % a.nl] * kLog2eD;
+                wait_phase(qfull + qi, qph, dead, &s_abort);
+                const unsigned char *qb = qbuf + (size_t)qi * rb;
 #pragma unroll
                 for (int hh = 0; hh < HPW; ++hh) {
                     m[hh] = -INFINITY;
@@ -283,157 +353,128 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
                         float x[VE];
-                        if (h < H) {
-                            const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(
-                                reinterpret_cast<const T *>(a.q) + seg_vec + (size_t)h * D +
-                                (v * LPR + c) * VE));
-                            Vec<T>::unpack(raw, x);
-                        }
+                        Vec<T>::unpack(*reinterpret_cast<const uint4 *>(qb + (size_t)h * D * sizeof(T) + (v * LPR + c) * 16), x);
 #pragma unroll
                         for (int i = 0; i < VE; ++i) {
-                            qf[hh][v * VE + i] = h < H ? x[i] * sc : 0.f;
+                            qf[hh][v * VE + i] = x[i] * sc;
                             acc[hh][v * VE + i] = 0.f;
                         }
                     }
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(qempty + qi);
+                qi ^= 1;
+                if (qi == 0) qph ^= 1u;
             }
-            const int r0 = (u - P[si]) * kUnitRows;
-            const int cnt = min(kUnitRows, n - r0);
+            const int cnt = min(UR, n + 1 - r0);  // rows of this unit, the appended row included
+            const int new_idx = n - r0;           // its index in the unit when 0 <= new_idx < UR
+            const bool seg_end = new_idx < UR;
+            float s[HPW][RPG];
+            const bool whole = cnt == UR;  // every row of the unit is valid (uniform over the CTA)
 
-            // ---- K item: logits of up to four rows --------------------------------------
+            // ---- K item: logits ---------------------------------------------------------------
             {
-                const int slot = it % a.nstages;
-                const uint32_t ph = (uint32_t)(it / a.nstages) & 1u;
-                if (!timed_out && !*(volatile int *)&s_abort && !mbar_wait(full + slot, ph)) {
-                    timed_out = true;
-                    atomicExch(&s_abort, 1);
-                }
-                const unsigned char *kb = ring + (size_t)slot * slot_bytes;
+                wait_phase(full + r.slot, r.phase, dead, &s_abort);
+                const unsigned char *kb = ring + (uint32_t)r.slot * slot_bytes;
+                const unsigned char *kl = kb + (uint32_t)g * rb + lane_off;
 #pragma unroll
-                for (int j = 0; j < kUnitRows / GPW; ++j) {
-                    const int rr = g + j * GPW;
+                for (int j = 0; j < RPG; ++j) {
 #pragma unroll
                     for (int hh = 0; hh < HPW; ++hh) {
-                        const int h = h0 + hh;
-                        float dot = 0.f;
-                        if (rr < cnt && h < H) {
-                            const unsigned char *row = kb + (size_t)rr * a.row_bytes + (size_t)h * D * sizeof(T);
+                        float d0 = 0.f, d1 = 0.f;
+                        if (whole || g + j * GPW < cnt) {
+                            const unsigned char *row = kl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
 #pragma unroll
                             for (int v = 0; v < NV; ++v) {
-                                const uint4 raw = *reinterpret_cast<const uint4 *>(row + (v * LPR + c) * 16);
                                 float x[VE];
-                                Vec<T>::unpack(raw, x);
+                                Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
 #pragma unroll
-                                for (int i = 0; i < VE; ++i) dot = fmaf(qf[hh][v * VE + i], x[i], dot);
+                                for (int i = 0; i < VE; i += 2) {
+                                    d0 = fmaf(qf[hh][v * VE + i], x[i], d0);
+                                    d1 = fmaf(qf[hh][v * VE + i + 1], x[i + 1], d1);
+                                }
                             }
                         }
-#pragma unroll
-                        for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                        s[hh][j] = dot;
+                        s[hh][j] = d0 + d1;
                     }
                 }
+#pragma unroll
+                for (int o = LPR / 2; o > 0; o >>= 1)
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j)
+#pragma unroll
+                        for (int hh = 0; hh < HPW; ++hh) s[hh][j] += __shfl_xor_sync(0xffffffffu, s[hh][j], o);
+                if (seg_end) {  // append: this warp's heads of the new K row go to cache row n
+                    const unsigned char *src = kb + (uint32_t)new_idx * rb + (uint32_t)h0 * D * sizeof(T);
+                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.ck) + (size_t)(off + n) * rb +
+                                         (size_t)h0 * D * sizeof(T);
+                    for (int x = lane; x < HPW * (int)(D * sizeof(T) / 16); x += 32)
+                        *reinterpret_cast<uint4 *>(dst + x * 16) = *reinterpret_cast<const uint4 *>(src + x * 16);
+                }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(empty + slot);
-                ++it;
+                if (lane == 0) mbar_arrive(empty + r.slot);
+                r.advance();
             }
-            // ---- V item: softmax update and accumulation ----------------------------------
+            // ---- V item: softmax update (one rescale per unit) and accumulation -------------------
             {
-                const int slot = it % a.nstages;
-                const uint32_t ph = (uint32_t)(it / a.nstages) & 1u;
-                if (!timed_out && !*(volatile int *)&s_abort && !mbar_wait(full + slot, ph)) {
-                    timed_out = true;
-                    atomicExch(&s_abort, 1);
-                }
-                const unsigned char *vb = ring + (size_t)slot * slot_bytes;
-#pragma unroll
-                for (int j = 0; j < kUnitRows / GPW; ++j) {
-                    const int rr = g + j * GPW;
-#pragma unroll
-                    for (int hh = 0; hh < HPW; ++hh) {
-                        const int h = h0 + hh;
-                        if (rr < cnt && h < H) {
-                            const float sv = s[hh][j];
-                            if (sv > m[hh]) {
-                                const float corr = exp2f(m[hh] - sv);
-                                l[hh] *= corr;
-#pragma unroll
-                                for (int i = 0; i < EPL; ++i) acc[hh][i] *= corr;
-                                m[hh] = sv;
-                            }
-                            const float p = exp2f(sv - m[hh]);
-                            l[hh] += p;
-                            const unsigned char *row = vb + (size_t)rr * a.row_bytes + (size_t)h * D * sizeof(T);
-#pragma unroll
-                            for (int v = 0; v < NV; ++v) {
-                                const uint4 raw = *reinterpret_cast<const uint4 *>(row + (v * LPR + c) * 16);
-                                float x[VE];
-                                Vec<T>::unpack(raw, x);
-#pragma unroll
-                                for (int i = 0; i < VE; ++i)
-                                    acc[hh][v * VE + i] = fmaf(p, x[i], acc[hh][v * VE + i]);
-                            }
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty + slot);
-                ++it;
-            }
-
-            const bool seg_end = (u == P[si + 1] - 1);
-            if (seg_end) {
-                // ---- the row appended this step: taken from the inputs, stored as row n -------
-                const size_t row_vec = (size_t)(a.row_offset[seg] + n) * H * D;
 #pragma unroll
                 for (int hh = 0; hh < HPW; ++hh) {
-                    const int h = h0 + hh;
-                    float dot = 0.f;
-                    uint4 vraw[NV];
-                    if (h < H) {
+                    float mx = m[hh];
 #pragma unroll
-                        for (int v = 0; v < NV; ++v) {
-                            const size_t e = seg_vec + (size_t)h * D + (v * LPR + c) * VE;
-                            const uint4 kraw = __ldg(reinterpret_cast<const uint4 *>(
-                                reinterpret_cast<const T *>(a.k_new) + e));
-                            vraw[v] = __ldg(reinterpret_cast<const uint4 *>(
-                                reinterpret_cast<const T *>(a.v_new) + e));
-                            if (g == 0) {
-                                const size_t d = row_vec + (size_t)h * D + (v * LPR + c) * VE;
-                                *reinterpret_cast<uint4 *>(reinterpret_cast<T *>(a.ck) + d) = kraw;
-                                *reinterpret_cast<uint4 *>(reinterpret_cast<T *>(a.cv) + d) = vraw[v];
-                            }
-                            float x[VE];
-                            Vec<T>::unpack(kraw, x);
-#pragma unroll
-                            for (int i = 0; i < VE; ++i) dot = fmaf(qf[hh][v * VE + i], x[i], dot);
-                        }
+                    for (int j = 0; j < RPG; ++j) {
+                        if (!(whole || g + j * GPW < cnt)) s[hh][j] = -INFINITY;
+                        mx = fmaxf(mx, s[hh][j]);
                     }
+                    // mx stays -inf only for a group that has seen no row yet; keep its state at zero
+                    const float corr = mx == -INFINITY ? 1.f : exp2f(m[hh] - mx);
+                    m[hh] = mx;
+                    float lsum = l[hh] * corr;
 #pragma unroll
-                    for (int o = LPR / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    if (g == 0 && h < H) {
-                        if (dot > m[hh]) {
-                            const float corr = exp2f(m[hh] - dot);
-                            l[hh] *= corr;
+                    for (int j = 0; j < RPG; ++j) {
+                        s[hh][j] = mx == -INFINITY ? 0.f : exp2f(s[hh][j] - mx);
+                        lsum += s[hh][j];
+                    }
+                    l[hh] = lsum;
 #pragma unroll
-                            for (int i = 0; i < EPL; ++i) acc[hh][i] *= corr;
-                            m[hh] = dot;
-                        }
-                        const float p = exp2f(dot - m[hh]);
-                        l[hh] += p;
+                    for (int i = 0; i < EPL; ++i) acc[hh][i] *= corr;
+                }
+                wait_phase(full + r.slot, r.phase, dead, &s_abort);
+                const unsigned char *vb = ring + (uint32_t)r.slot * slot_bytes;
+                const unsigned char *vl = vb + (uint32_t)g * rb + lane_off;
 #pragma unroll
-                        for (int v = 0; v < NV; ++v) {
-                            float x[VE];
-                            Vec<T>::unpack(vraw[v], x);
+                for (int j = 0; j < RPG; ++j) {
 #pragma unroll
-                            for (int i = 0; i < VE; ++i)
-                                acc[hh][v * VE + i] = fmaf(p, x[i], acc[hh][v * VE + i]);
+                    for (int hh = 0; hh < HPW; ++hh) {
+                        if (whole || g + j * GPW < cnt) {
+                            const float pj = s[hh][j];
+                            const unsigned char *row = vl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
+#pragma unroll
+                            for (int v = 0; v < NV; ++v) {
+                                float x[VE];
+                                Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
+#pragma unroll
+                                for (int i = 0; i < VE; ++i)
+                                    acc[hh][v * VE + i] = fmaf(pj, x[i], acc[hh][v * VE + i]);
+                            }
                         }
                     }
                 }
+                if (seg_end) {
+                    const unsigned char *src = vb + (uint32_t)new_idx * rb + (uint32_t)h0 * D * sizeof(T);
+                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.cv) + (size_t)(off + n) * rb +
+                                         (size_t)h0 * D * sizeof(T);
+                    for (int x = lane; x < HPW * (int)(D * sizeof(T) / 16); x += 32)
+                        *reinterpret_cast<uint4 *>(dst + x * 16) = *reinterpret_cast<const uint4 *>(src + x * 16);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + r.slot);
+                r.advance();
             }
+            r0 += UR;
+
             if (seg_end || u == u1 - 1) {
                 // ---- close this CTA's piece of the segment ---------------------------------------
-                const int c_first = unit_owner(P[si], G, U), c_last = unit_owner(P[si + 1] - 1, G, U);
+                const int c_first = unit_owner(P[si], upc, rem), c_last = unit_owner(P[si + 1] - 1, upc, rem);
                 const int ncontrib = c_last - c_first + 1;
 #pragma unroll
                 for (int hh = 0; hh < HPW; ++hh) {
@@ -480,84 +521,118 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                         }
                     }
                 }
-                if (ncontrib > 1) {
-                    __threadfence();
-                    consumer_barrier(NW * 32);
-                    if (tid == 0) {
-                        __threadfence();
-                        const int old = atomicAdd(a.arrive + seg, 1);
-                        s_flag = (old == ncontrib - 1);
-                    }
-                    consumer_barrier(NW * 32);
-                    if (s_flag) {
-                        __threadfence();
-                        for (int hh = 0; hh < HPW; ++hh) {
-                            const int h = h0 + hh;
-                            if (h >= H) continue;
-                            float M = -INFINITY;
-                            for (int cc = c_first; cc <= c_last; ++cc)
-                                M = fmaxf(M, __ldcg(a.scratch + ((size_t)(cc + si) * H + h) * kSlotStride + D));
-                            float z = 0.f, o[D / 32];
-#pragma unroll
-                            for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
-                            for (int cc = c_first; cc <= c_last; ++cc) {
-                                const float *slot = a.scratch + ((size_t)(cc + si) * H + h) * kSlotStride;
-                                const float w = exp2f(__ldcg(slot + D) - M);
-                                z += w * __ldcg(slot + D + 1);
-#pragma unroll
-                                for (int i = 0; i < D / 32; ++i) o[i] += w * __ldcg(slot + lane + 32 * i);
-                            }
-                            const float inv = 1.f / z;
-                            T *dst = reinterpret_cast<T *>(a.out) + seg_vec + (size_t)h * D;
-#pragma unroll
-                            for (int i = 0; i < D / 32; ++i) dst[lane + 32 * i] = from_float<T>(o[i] * inv);
-                        }
-                        consumer_barrier(NW * 32);
-                        if (tid == 0) a.arrive[seg] = 0;
-                    }
-                }
-                fresh = true;
+                piece_start = true;
             }
         }
-        if (timed_out && lane == 0) raise_status(a.dev_status, 0, PKV_DEV_TIMEOUT);
+
+        if (dead && lane == 0) raise_status(a.dev_status, 0, PKV_DEV_TIMEOUT);
     }
 
-    // ---- last CTA of the grid: every CTA has read the lengths, so they can grow ----------
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        const int old = atomicAdd(a.arrive + a.nseg_total, 1);
-        s_flag = (old == (int)gridDim.x - 1);
-    }
-    __syncthreads();
-    if (s_flag) {
-        for (int si = tid; si < a.nact; si += blockDim.x) {
-            if (nlen[si] < 0) continue;
-            const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-            a.len[seg] = nlen[si] + 1;
-        }
-        if (tid == 0) a.arrive[a.nseg_total] = 0;
-    }
 }
+
+// Merge kernel: one warp per (head, active segment), launched as a programmatic dependent of
+// the stream kernel.  For a segment split over several CTAs it combines their partials with
+// every load of a batch in flight at once (three round trips for up to 16 contributors); for
+// every segment that took a row, the warp of head 0 bumps len.
+template <typename T, int D>
+__global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
+{
+    constexpr int kSlotStride = D + 4;
+    constexpr int KB = 16;  // contributors per batch
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
+    const int h = blockIdx.x, si = blockIdx.y, lane = threadIdx.x;
+    const int *P = a.plan + 4;
+    const int n = a.plan[5 + a.nact + si];
+    if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
+    const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+    const int upc = a.plan[2], rem = a.plan[3];
+    const int c_first = unit_owner(P[si], upc, rem), c_last = unit_owner(P[si + 1] - 1, upc, rem);
+    const int ncontrib = c_last - c_first + 1;
+    if (h == 0 && lane == 0) a.len[seg] = n + 1;
+    if (ncontrib == 1) return;
+    const size_t cstride = (size_t)a.H * kSlotStride;
+    const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;
+    float mloc = -INFINITY, zloc = 0.f;
+    for (int k = lane; k < ncontrib; k += 32) {  // online over this lane's contributors
+        const float mk = base[k * cstride + D], lk = base[k * cstride + D + 1];
+        const float mn = fmaxf(mloc, mk);
+        zloc = zloc * exp2f(mloc - mn) + lk * exp2f(mk - mn);
+        mloc = mn;
+    }
+    const float M = warp_max(mloc);
+    const float z = warp_sum(mloc == -INFINITY ? 0.f : zloc * exp2f(mloc - M));
+    float o[D / 32];
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
+    for (int k0 = 0; k0 < ncontrib; k0 += KB) {
+        float w[KB], x[KB][D / 32];
+#pragma unroll
+        for (int kk = 0; kk < KB; ++kk) {
+            const float *sl = base + min(k0 + kk, ncontrib - 1) * cstride;
+            w[kk] = sl[D];
+#pragma unroll
+            for (int i = 0; i < D / 32; ++i) x[kk][i] = sl[lane + 32 * i];
+        }
+#pragma unroll
+        for (int kk = 0; kk < KB; ++kk) {
+            if (k0 + kk < ncontrib) {
+                const float ww = exp2f(w[kk] - M);
+#pragma unroll
+                for (int i = 0; i < D / 32; ++i) o[i] = fmaf(ww, x[kk][i], o[i]);
+            }
+        }
+    }
+    const float inv = 1.f / z;
+    T *dst = reinterpret_cast<T *>(a.out) + ((size_t)seg * a.H + h) * D;
+#pragma unroll
+    for (int i = 0; i < D / 32; ++i) dst[lane + 32 * i] = from_float<T>(o[i] * inv);
+}
+
+static size_t plan_bytes(int nact) { return round_up((size_t)(5 + 2 * nact) * sizeof(int), kWsAlign); }
 
 size_t decode_stream_ws_bytes(const pkv_shape *s)
 {
-    size_t slots = 256 + (size_t)s->batch * s->layers;
-    return round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
+    size_t nseg = (size_t)s->batch * s->layers;
+    size_t slots = 256 + nseg;
+    return plan_bytes((int)(nseg < (size_t)kMaxActive ? nseg : kMaxActive)) +
+           round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
 }
 
-template <typename T, int D, int LPR, int HPW, int MAXT>
+static size_t stream_smem_bytes(int nstages, int ur, uint32_t rb, int nact)
+{
+    return (size_t)nstages * ur * rb + 2 * (size_t)rb + (2 * kMaxStages + 4) * sizeof(uint64_t) +
+           (size_t)nact * sizeof(int64_t) + (size_t)(2 * nact + 1) * sizeof(int) + 32;
+}
+
+template <typename T, int D, int LPR, int HPW, int UR, int MAXT>
 static int launch_variant(const DecodeArgs &a, int sms, cudaStream_t st)
 {
     static bool done[64] = {};
-    const size_t slot_bytes = (size_t)kUnitRows * a.row_bytes;
-    const size_t smem = (size_t)a.nstages * slot_bytes + 2 * kMaxStages * sizeof(uint64_t) +
-                        (size_t)(2 * a.nact + 1) * sizeof(int) + 16;
     if ((a.nwarps + 1) * 32 > MAXT) return -1;
-    int rc = ensure_dynamic_smem((const void *)decode_stream_kernel<T, D, LPR, HPW, MAXT>, kDynSmemMax, done);
+    int rc = ensure_dynamic_smem((const void *)decode_stream_kernel<T, D, LPR, HPW, UR, MAXT>, kDynSmemMax, done);
     if (rc != PKV_OK) return rc;
-    decode_stream_kernel<T, D, LPR, HPW, MAXT><<<sms, (a.nwarps + 1) * 32, smem, st>>>(a);
-    return check_launch("decode_stream_kernel");
+    decode_stream_kernel<T, D, LPR, HPW, UR, MAXT>
+        <<<sms, (a.nwarps + 1) * 32, stream_smem_bytes(a.nstages, UR, a.row_bytes, a.nact), st>>>(a);
+    rc = check_launch("decode_stream_kernel");
+    if (rc != PKV_OK) return rc;
+    // The merge kernel is a programmatic dependent: it may be set up while the stream kernel
+    // runs and starts past its griddepcontrol.wait once that grid has completed.
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(a.H, a.nact);
+    cfg.blockDim = dim3(32);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D>, a);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "decode_finish_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
 
 // Returns PKV_OK, an error, or -1 when this shape is outside what the streaming kernel covers.
@@ -565,17 +640,20 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
                          const void *vn, const float *scale, int lb, int le, void *out,
                          int32_t *dev_status, void *ws, cudaStream_t st)
 {
-    if (!c->arrive) return -1;
     const int H = s->heads, D = s->head_dim, nl = le - lb, nact = s->batch * nl;
     if (nact > kMaxActive || H > 64) return -1;
     const size_t es = esize(s);
     const uint32_t row_bytes = (uint32_t)((size_t)H * D * es);
-    const size_t slot_bytes = (size_t)kUnitRows * row_bytes;
-    const size_t meta = 2 * kMaxStages * sizeof(uint64_t) + (size_t)(2 * nact + 1) * sizeof(int) + 256;
-    const size_t budget = kDynSmemMax - meta;
-    int nstages = (int)(budget / slot_bytes);
-    if (nstages > kMaxStages) nstages = kMaxStages;
-    if (nstages < 3) return -1;
+    int ur = 0, nstages = 0;
+    for (int cand = 8; cand >= 4 && !ur; cand >>= 1) {
+        int ns = kMaxStages;
+        while (ns >= 3 && stream_smem_bytes(ns, cand, row_bytes, nact) > (size_t)kDynSmemMax) --ns;
+        if (ns >= 3) {
+            ur = cand;
+            nstages = ns;
+        }
+    }
+    if (!ur) return -1;
 
     static int sm_count[64] = {};
     int dev = 0;
@@ -593,47 +671,58 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
 
     DecodeArgs a;
     a.q = q; a.k_new = kn; a.v_new = vn; a.ck = c->k; a.cv = c->v; a.out = out;
-    a.row_offset = c->row_offset; a.len = c->len; a.cap = c->cap; a.arrive = c->arrive;
-    a.layer_scale = scale; a.scratch = (float *)ws; a.dev_status = dev_status;
+    a.row_offset = c->row_offset; a.len = c->len; a.cap = c->cap;
+    a.layer_scale = scale; a.dev_status = dev_status;
+    a.plan = (int *)ws;
+    a.scratch = (float *)((unsigned char *)ws + plan_bytes(nact));
     a.L = s->layers; a.H = H; a.layer_begin = lb; a.nl = nl; a.nact = nact;
     a.nseg_total = s->batch * s->layers; a.nstages = nstages; a.row_bytes = row_bytes;
+    a.total_cap_rows = c->total_cap_rows;
 
     const bool bf = s->dtype == PKV_BF16;
     const int vec_per_head = D / (int)(16 / es);
-    // (lanes per row, heads per warp): fewer, fatter warps once H > 16 so that the register
-    // file of each SM sub-partition holds the per-head state without spilling.
-    int lpr = 8, hpw = H <= 16 ? 1 : 4;
-    if (H > 32 && vec_per_head >= 16) lpr = 16;
+    // (lanes per row, heads per warp): at most 17 warps, and few enough registers of per-head
+    // state that each SM sub-partition's register file holds its warps.
+    int lpr = 8, hpw = H <= 16 ? 1 : (H <= 32 ? 2 : 4);
+    if (H > 16 && vec_per_head >= 16) lpr = 16;
     if (const char *env = getenv("PKV_DECODE_VARIANT")) {
         int code = atoi(env);
         if (code > 0) { lpr = code / 10; hpw = code % 10; }
     }
-    if (vec_per_head < lpr) return -1;
-    a.nwarps = (H + hpw - 1) / hpw;
-#define PKV_V(T, DD, LPR, HPW, MAXT) \
-    if (lpr == LPR && hpw == HPW && (a.nwarps + 1) * 32 <= MAXT) \
-        return launch_variant<T, DD, LPR, HPW, MAXT>(a, sms, st)
-#define PKV_FAMILY(T, DD)            \
-    PKV_V(T, DD, 8, 1, 544);         \
-    PKV_V(T, DD, 8, 2, 544);         \
-    PKV_V(T, DD, 8, 4, 288);         \
-    PKV_V(T, DD, 8, 4, 544)
+    if (vec_per_head < lpr || H % hpw != 0) return -1;
+    a.nwarps = H / hpw;
+#define PKV_V(T, DD, LPR, HPW, UR, MAXT)                                       \
+    if (lpr == LPR && hpw == HPW && ur == UR && (a.nwarps + 1) * 32 <= MAXT) \
+        return launch_variant<T, DD, LPR, HPW, UR, MAXT>(a, sms, st)
+#define PKV_FAMILY(T, DD)        \
+    PKV_V(T, DD, 8, 1, 8, 544);  \
+    PKV_V(T, DD, 8, 2, 8, 544);  \
+    PKV_V(T, DD, 8, 4, 8, 288);  \
+    PKV_V(T, DD, 8, 4, 8, 544);  \
+    PKV_V(T, DD, 8, 1, 4, 544);  \
+    PKV_V(T, DD, 8, 2, 4, 544);  \
+    PKV_V(T, DD, 8, 4, 4, 288);  \
+    PKV_V(T, DD, 8, 4, 4, 544)
+#define PKV_WIDE(T, DD)           \
+    PKV_V(T, DD, 16, 2, 8, 544);  \
+    PKV_V(T, DD, 16, 4, 8, 288);  \
+    PKV_V(T, DD, 16, 4, 8, 544);  \
+    PKV_V(T, DD, 16, 2, 4, 544);  \
+    PKV_V(T, DD, 16, 4, 4, 288);  \
+    PKV_V(T, DD, 16, 4, 4, 544)
     if (bf && D == 128) {
         PKV_FAMILY(__nv_bfloat16, 128);
-        PKV_V(__nv_bfloat16, 128, 16, 2, 544);
-        PKV_V(__nv_bfloat16, 128, 16, 4, 288);
-        PKV_V(__nv_bfloat16, 128, 16, 4, 544);
+        PKV_WIDE(__nv_bfloat16, 128);
     } else if (bf && D == 64) {
         PKV_FAMILY(__nv_bfloat16, 64);
     } else if (!bf && D == 128) {
         PKV_FAMILY(float, 128);
-        PKV_V(float, 128, 16, 2, 544);
-        PKV_V(float, 128, 16, 4, 288);
-        PKV_V(float, 128, 16, 4, 544);
+        PKV_WIDE(float, 128);
     } else if (!bf && D == 64) {
         PKV_FAMILY(float, 64);
-        PKV_V(float, 64, 16, 4, 544);
+        PKV_WIDE(float, 64);
     }
+#undef PKV_WIDE
 #undef PKV_FAMILY
 #undef PKV_V
     return -1;
