@@ -195,35 +195,43 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     w = wl.WORKLOADS[args.workload]
-    # Ranks hold different samples of the same workload (batch sharding, no exchange).
-    samples = [rank * w.B + b for b in range(w.B)]
-    q, k, v = wl.make_prompt(w, dev, samples=samples)
     scale = wl.layer_scale(w)
     budget = w.budget_rows()
-    s = Session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T, max_budget_rows=budget,
-                device=dev)
-    s.budget.fill_(budget)
+    # Inputs larger than L2: R independent prompts (replicas) are run interleaved, each as its own
+    # batch-B call, so that between two calls on one prompt's data at least 256 MiB of other
+    # prompts' K/V has passed through the 126 MB L2.  No flush kernel sits in the timed region.
+    retained_bytes = 2 * w.B * budget * w.row_bytes
+    R = max(1, min(8, 1 + -(-(256 << 20) // retained_bytes))) if retained_bytes < (256 << 20) else 1
+    # Ranks hold different samples of the same workload (batch sharding, no exchange).
+    reps = []
+    for r in range(R):
+        samples = [(rank * R + r) * w.B + b for b in range(w.B)]
+        q, k, v = wl.make_prompt(w, dev, samples=samples)
+        s = Session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T, max_budget_rows=budget,
+                    device=dev)
+        s.budget.fill_(budget)
+        reps.append((s, q, k, v))
+    s, q, k, v = reps[0]
     n_pool = 8
-    pool = [wl.make_decode_inputs(w, t, dev, samples=samples) for t in range(n_pool)]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
+    pool = [wl.make_decode_inputs(w, t, dev, samples=list(range(w.B))) for t in range(n_pool)]
     stream = torch.cuda.current_stream()
 
-    def step(events=None):
-        """One pass of the whole path; optionally records (start, end) CUDA events per stage."""
+    def step(events):
+        """One pass of the whole path for each of the R prompts; one CUDA-event pair per stage."""
         def timed(fn, tag):
-            if events is None:
-                fn()
-                return
-            flush.zero_()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream); fn(); b.record(stream)
             events.append((tag, a, b))
-        timed(lambda: s.score(q, k), "score")
-        timed(lambda: s.search(None, tol=w.tol), "search")
-        timed(lambda: s.compact(k, v), "compact")
-        for t in range(w.T):
-            qd, kn, vn = pool[t % n_pool]
-            timed(lambda: s.decode(qd, kn, vn), "decode")
+        timed(lambda: [ss.score(qq, kk) for ss, qq, kk, vv in reps], "score")
+        timed(lambda: [ss.search(None, tol=w.tol) for ss, qq, kk, vv in reps], "search")
+        timed(lambda: [ss.compact(kk, vv) for ss, qq, kk, vv in reps], "compact")
+
+        def decode_all():
+            for t in range(w.T):
+                qd, kn, vn = pool[t % n_pool]
+                for ss, _, _, _ in reps:
+                    ss.decode(qd, kn, vn)
+        timed(decode_all, "decode")
 
     def barrier():
         torch.cuda.synchronize()
@@ -246,14 +254,16 @@ def run_ours(args):
     barrier()
     wall = time.perf_counter() - wall0
     clocks = sampler.stop() if rank == 0 else None
-    assert s.status.cpu().tolist() == [0] * w.B, "device status raised"
+    for ss, _, _, _ in reps:
+        assert ss.status.cpu().tolist() == [0] * w.B, "device status raised"
 
+    # per prompt: each stage's event time divided by the R prompts it covered
     stage_ms = {"score": 0.0, "search": 0.0, "compact": 0.0, "decode": 0.0}
     for ev in all_events:
         for tag, a, b in ev:
             stage_ms[tag] += a.elapsed_time(b)
     for kx in stage_ms:
-        stage_ms[kx] /= args.steps
+        stage_ms[kx] /= args.steps * R
     step_ms = sum(stage_ms.values())
     t_max = torch.tensor([step_ms], dtype=torch.float64, device=dev)
     if world > 1:
@@ -295,9 +305,12 @@ def run_ours(args):
         "config": {"workload": w.name, "batch": w.B, "layers": w.L, "heads": w.H, "head_dim": w.D,
                    "prompt_len": w.N, "budget_rows": budget, "decode_steps": w.T,
                    "parallelism": "batch-sharded x%d, no collective" % world,
-                   "l2": "256 MiB write between timed stages (outside the event pairs)",
-                   "timing": "sum of CUDA-event stage times; wall %.1f ms/step incl. flushes"
-                             % (1e3 * wall / args.steps)},
+                   "prompts_interleaved": R,
+                   "l2": "inputs larger than L2: %d independent prompts interleaved call by call, so "
+                         ">= 256 MiB of other K/V passes between two calls on one prompt" % R,
+                   "timing": "one CUDA-event pair per stage over all %d prompts; ms_per_step and "
+                             "stages_ms are per prompt; wall %.2f ms per prompt"
+                             % (R, 1e3 * wall / (args.steps * R))},
         "stages_ms": stage_ms,
         "decode_attn": {"gbs": dec_gbs, "pct_of_8tbs": 100 * dec_gbs / NOMINAL_HBM_GBS,
                         "pct_of_measured_copy": 100 * dec_gbs / hbm_peak,
@@ -306,11 +319,11 @@ def run_ours(args):
                      "compact_gbs": compact_bytes / (stage_ms["compact"] * 1e-3) / 1e9,
                      "score_tensor_util_vs_burst": causal_flop * 2 / (stage_ms["score"] * 1e-3) / (tf_peak * 1e12),
                      "target_ms_strict": causal_flop / (0.5 * tf_peak * 1e12) * 1e3},
-        "roofline": {"bound": "hbm", "kernel": "decode attention (one call = one decode step)",
+        "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel + its merge kernel (one decode call, launch gaps included)",
                      "achieved": dec_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": dec_gbs / hbm_peak,
                      "peak_kind": "of " + peak_kind, "traffic": None,
                      "bytes_per_launch": dec_bytes / w.T, "us_per_launch": 1e3 * stage_ms["decode"] / w.T},
-        "gpu_launches": args.steps * LAUNCHES_PER_STEP(w),
+        "gpu_launches": args.steps * R * LAUNCHES_PER_STEP(w),
         "clocks": clocks,
     }
     if e2e is not None:
@@ -319,7 +332,7 @@ def run_ours(args):
                        "note": "host pinned Q,K,V and per-token q,k,v copied in, outputs copied out, "
                                "wall clock, no L2 flush"}
     if world == 1 and not args.no_cpu_baseline:
-        v_cpu, desc, spent = time_oracle_sample(w, score_layers=4, decode_steps=(0, 1))
+        v_cpu, desc, spent = time_oracle_sample(w, score_layers=min(w.L, 16), decode_steps=(0, 1, 2, 3))
         line["cpu_baseline"] = {"value": v_cpu, "unit": "tok/s", "cores": 1, "kind": "oracle",
                                 "sample": desc, "seconds": spent}
     print(json.dumps(line))
@@ -329,7 +342,7 @@ def run_ours(args):
 
 def LAUNCHES_PER_STEP(w):
     # score: lse + column sums + head mean; search: status clear + sort/scan + bisection;
-    # compact: plan + gather; decode: partial + merge per token
+    # compact: plan + gather; decode: stream + merge per token
     return 3 + 3 + 2 + 2 * w.T
 
 

@@ -35,9 +35,9 @@ struct DecodeArgs {
     const int32_t *cap;
     const float *layer_scale;
     float *scratch;   // partial slots
-    int *plan;        // [4 + (nact + 1) + nact]: U, G, units per CTA, remainder; unit prefix; rows
     int32_t *dev_status;
     int L, H, layer_begin, nl, nact, nseg_total, nstages, nwarps;
+    int unit_rows, grid;  // rows per unit and CTAs of the stream kernel (the merge kernel re-derives its plan)
     uint32_t row_bytes;
     int64_t total_cap_rows;
 };
@@ -143,6 +143,17 @@ __device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, bool 
     }
 }
 
+// Rows of active segment si that this step attends over besides the appended one, or -1
+// when the segment cannot take another row (full, never compacted, or outside the cache).
+__device__ __forceinline__ int segment_rows(const DecodeArgs &a, int si, int64_t *off_out = nullptr)
+{
+    const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+    const int ln = a.len[seg], cp = a.cap[seg];
+    const int64_t off = a.row_offset[seg];
+    if (off_out) *off_out = off;
+    return (ln >= 1 && ln < cp && off >= 0 && off + cp <= a.total_cap_rows) ? ln : -1;
+}
+
 struct Ring {
     int slot, nstages;
     uint32_t phase;
@@ -201,13 +212,11 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         P[0] = 0;
     }
     for (int si = tid; si < a.nact; si += blockDim.x) {
-        const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-        const int ln = a.len[seg], cp = a.cap[seg];
-        const int64_t off = a.row_offset[seg];
-        const bool ok = ln >= 1 && ln < cp && off >= 0 && off + cp <= a.total_cap_rows;
-        seg_n[si] = ok ? ln : -1;
+        int64_t off;
+        const int rows = segment_rows(a, si, &off);
+        seg_n[si] = rows;
         seg_off[si] = off;
-        P[si + 1] = ok ? (ln + UR) / UR : 0;  // ceil((ln + 1) / UR): the appended row is the last row
+        P[si + 1] = rows >= 0 ? (rows + UR) / UR : 0;  // ceil((rows + 1) / UR): the appended row is the last row
     }
     __syncthreads();
     if (warp == 0) {
@@ -242,13 +251,6 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
     const int upc = G > 0 ? U / G : 0, rem = G > 0 ? U - upc * G : 0;
     // The merge kernel may be scheduled from here on; it still waits for this grid to finish.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (cta == 0) {  // the plan, for the merge kernel
-        if (tid == 0) {
-            a.plan[0] = U; a.plan[1] = G; a.plan[2] = upc; a.plan[3] = rem;
-        }
-        for (int i = tid; i <= a.nact; i += blockDim.x) a.plan[4 + i] = P[i];
-        for (int i = tid; i < a.nact; i += blockDim.x) a.plan[5 + a.nact + i] = seg_n[i];
-    }
     if (cta < G) {
         u0 = first_unit(cta, upc, rem);
         u1 = first_unit(cta + 1, upc, rem);
@@ -531,52 +533,82 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 }
 
 // Merge kernel: one warp per (head, active segment), launched as a programmatic dependent of
-// the stream kernel.  For a segment split over several CTAs it combines their partials with
-// every load of a batch in flight at once (three round trips for up to 16 contributors); for
-// every segment that took a row, the warp of head 0 bumps len.
+// the stream kernel.  Before it waits for that grid it rebuilds the unit plan from the
+// lengths (which the stream kernel only reads), so that afterwards one round trip fetches
+// the partials of up to 16 contributing CTAs at once.  For a segment split over several CTAs
+// it combines their partials; for every segment that took a row, the warp of head 0 bumps len.
 template <typename T, int D>
 __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
 {
     constexpr int kSlotStride = D + 4;
     constexpr int KB = 16;  // contributors per batch
-    asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
     const int h = blockIdx.x, si = blockIdx.y, lane = threadIdx.x;
-    const int *P = a.plan + 4;
-    const int n = a.plan[5 + a.nact + si];
-    if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
+
+    // ---- same plan as the stream kernel: units before this segment, in it, and in total ------
+    int before = 0, mine = 0, total = 0, n = -1;
+    for (int base = 0; base < a.nact; base += 32) {
+        const int i = base + lane;
+        int units = 0;
+        if (i < a.nact) {
+            const int rows = segment_rows(a, i);
+            units = rows >= 0 ? (rows + a.unit_rows) / a.unit_rows : 0;
+            if (i == si) n = rows;
+        }
+        int incl = units;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (si >= base && si < base + 32) {
+            before = total + __shfl_sync(0xffffffffu, incl - units, si - base);
+            mine = __shfl_sync(0xffffffffu, units, si - base);
+        }
+        total += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    n = __shfl_sync(0xffffffffu, n, si & 31);
+    const int G = a.grid < total ? a.grid : total;
+    const int upc = G > 0 ? total / G : 0, rem = G > 0 ? total - upc * G : 0;
     const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-    const int upc = a.plan[2], rem = a.plan[3];
-    const int c_first = unit_owner(P[si], upc, rem), c_last = unit_owner(P[si + 1] - 1, upc, rem);
-    const int ncontrib = c_last - c_first + 1;
+    int c_first = 0, ncontrib = 0;
+    if (n >= 0) {
+        c_first = unit_owner(before, upc, rem);
+        ncontrib = unit_owner(before + mine - 1, upc, rem) - c_first + 1;
+    }
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
+    if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
     if (h == 0 && lane == 0) a.len[seg] = n + 1;
     if (ncontrib == 1) return;
     const size_t cstride = (size_t)a.H * kSlotStride;
     const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;
-    float mloc = -INFINITY, zloc = 0.f;
-    for (int k = lane; k < ncontrib; k += 32) {  // online over this lane's contributors
-        const float mk = base[k * cstride + D], lk = base[k * cstride + D + 1];
-        const float mn = fmaxf(mloc, mk);
-        zloc = zloc * exp2f(mloc - mn) + lk * exp2f(mk - mn);
-        mloc = mn;
-    }
-    const float M = warp_max(mloc);
-    const float z = warp_sum(mloc == -INFINITY ? 0.f : zloc * exp2f(mloc - M));
-    float o[D / 32];
+    float M = -INFINITY, z = 0.f, o[D / 32];
 #pragma unroll
     for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
     for (int k0 = 0; k0 < ncontrib; k0 += KB) {
-        float w[KB], x[KB][D / 32];
+        float w[KB], ls[KB], x[KB][D / 32];
 #pragma unroll
-        for (int kk = 0; kk < KB; ++kk) {
+        for (int kk = 0; kk < KB; ++kk) {  // every load of the batch is in flight before any use
             const float *sl = base + min(k0 + kk, ncontrib - 1) * cstride;
             w[kk] = sl[D];
+            ls[kk] = sl[D + 1];
 #pragma unroll
             for (int i = 0; i < D / 32; ++i) x[kk][i] = sl[lane + 32 * i];
         }
+        float mb = M;
+#pragma unroll
+        for (int kk = 0; kk < KB; ++kk)
+            if (k0 + kk < ncontrib) mb = fmaxf(mb, w[kk]);
+        const float corr = M == -INFINITY ? 0.f : exp2f(M - mb);
+        z *= corr;
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) o[i] *= corr;
+        M = mb;
 #pragma unroll
         for (int kk = 0; kk < KB; ++kk) {
             if (k0 + kk < ncontrib) {
                 const float ww = exp2f(w[kk] - M);
+                z = fmaf(ww, ls[kk], z);
 #pragma unroll
                 for (int i = 0; i < D / 32; ++i) o[i] = fmaf(ww, x[kk][i], o[i]);
             }
@@ -588,14 +620,11 @@ __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
     for (int i = 0; i < D / 32; ++i) dst[lane + 32 * i] = from_float<T>(o[i] * inv);
 }
 
-static size_t plan_bytes(int nact) { return round_up((size_t)(5 + 2 * nact) * sizeof(int), kWsAlign); }
-
 size_t decode_stream_ws_bytes(const pkv_shape *s)
 {
     size_t nseg = (size_t)s->batch * s->layers;
     size_t slots = 256 + nseg;
-    return plan_bytes((int)(nseg < (size_t)kMaxActive ? nseg : kMaxActive)) +
-           round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
+    return round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
 }
 
 static size_t stream_smem_bytes(int nstages, int ur, uint32_t rb, int nact)
@@ -673,11 +702,12 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     a.q = q; a.k_new = kn; a.v_new = vn; a.ck = c->k; a.cv = c->v; a.out = out;
     a.row_offset = c->row_offset; a.len = c->len; a.cap = c->cap;
     a.layer_scale = scale; a.dev_status = dev_status;
-    a.plan = (int *)ws;
-    a.scratch = (float *)((unsigned char *)ws + plan_bytes(nact));
+    a.scratch = (float *)ws;
     a.L = s->layers; a.H = H; a.layer_begin = lb; a.nl = nl; a.nact = nact;
     a.nseg_total = s->batch * s->layers; a.nstages = nstages; a.row_bytes = row_bytes;
     a.total_cap_rows = c->total_cap_rows;
+    a.unit_rows = ur;
+    a.grid = sms;
 
     const bool bf = s->dtype == PKV_BF16;
     const int vec_per_head = D / (int)(16 / es);
