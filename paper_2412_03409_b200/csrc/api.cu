@@ -56,11 +56,15 @@ int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const voi
                     cudaStream_t st);
 bool score_tc_usable(const pkv_shape *s, const void *q, pkv_strides qs, const void *k, pkv_strides ks);
 
+size_t score_tc_ws_bytes(const pkv_shape *s);
+
 static size_t score_ws_bytes(const pkv_shape *s)
 {
-    // per-head column sums + per-query log-sum-exp, both [B, L, H, N] fp32
+    // per-head column sums + per-query log-sum-exp, both [B, L, H, N] fp32; the tensor-core
+    // path pads the second to whole 128-query tiles
     size_t per = (size_t)s->batch * s->layers * s->heads * s->prompt_len * sizeof(float);
-    return round_up(2 * per, kWsAlign);
+    size_t simt = round_up(2 * per, kWsAlign), tc = score_tc_ws_bytes(s);
+    return simt > tc ? simt : tc;
 }
 
 // Gini coefficient from the descending cumulative sums.  The Lorenz curve over
@@ -124,8 +128,10 @@ extern "C" int prefixkv_score(const pkv_shape *shape, const void *q, pkv_strides
     if (!ws || !aligned(ws, kWsAlign) || ws_bytes < score_ws_bytes(shape)) return PKV_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (shape->dtype == PKV_BF16) {
-        if (score_tc_usable(shape, q, qs, k, ks))
-            return launch_score_tc(shape, q, qs, k, ks, layer_scale, lse, scores, ws, stream);
+        if (score_tc_usable(shape, q, qs, k, ks)) {
+            int rc = launch_score_tc(shape, q, qs, k, ks, layer_scale, lse, scores, ws, stream);
+            if (rc >= 0) return rc;  // -1: layout not expressible as a tensor map, use the FMA path
+        }
         if (shape->head_dim == 64)
             return launch_score_simt<__nv_bfloat16, 64>(shape, q, qs, k, ks, layer_scale, lse, scores,
                                                         ws, stream);

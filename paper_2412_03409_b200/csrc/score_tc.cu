@@ -1,17 +1,477 @@
-// Importance score (Sec. 3.2), tensor-core path for bf16 inputs (tcgen05 / TMEM / TMA).
+// Importance score (Sec. 3.2), tensor-core path for bf16 inputs.
+//
+//   pass 1: per query m, log2-sum-exp of the scaled causal logits over keys j <= m
+//   pass 2: per key n, sum over queries m >= n of exp2(logit - lse[m])
+//   then the mean over heads in index order (shared with the FP32 path)
+//
+// Both passes walk 128 x 128 logit tiles of one (sample, layer, head).  The tile is one
+// tcgen05.mma chain (M = N = 128, K = 16 x D/16) whose operands TMA stages in shared memory
+// with the 128-byte swizzle and whose fp32 accumulator lives in tensor memory.  The operand
+// that stays for a whole work item supplies the accumulator's lanes: queries in pass 1, so a
+// thread owns one query row and keeps its running max / sum in registers; keys in pass 2, so
+// a thread owns one key and its column sum needs no cross-thread reduction or atomics.
+//
+// Roles per CTA (192 threads): warp 0 lane 0 issues TMA, warp 1 owns tensor memory and its
+// lane 0 issues the MMAs, warps 2-5 read the accumulator (tcgen05.ld, one TMEM lane quarter
+// per warp) and do the exponentials.  Two accumulators alternate so that the MMAs of tile
+// j + 1 overlap the exponentials of tile j; two CTAs share an SM.  Every mbarrier wait is
+// bounded: when one runs out the CTA stops waiting, reports PKV_DEV_TIMEOUT and still
+// releases its tensor memory.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace pkv {
 
-bool score_tc_usable(const pkv_shape *, const void *, pkv_strides, const void *, pkv_strides)
+namespace {
+
+constexpr int TT = 128;            // tile side
+constexpr int kStagesB = 2;        // streamed-operand stages
+constexpr uint32_t kSpin = 1u << 22;
+constexpr float kLog2eT = 1.4426950408889634f;
+
+struct ScoreArgs {
+    const float *layer_scale;
+    float *lse2;     // [B*L*H][Npad] log2-sum-exp of scaled logits, +inf beyond N
+    float *partial;  // [B*L*H][N] per-head column sums
+    int32_t *abort_word;  // device word set when a bounded wait runs out (may be null)
+    int L, H, N, Npad, tiles, nseg;
+};
+
+__device__ __forceinline__ uint32_t saddr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bar_init(uint64_t *bar, uint32_t count)
 {
-    return false;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(saddr(bar)), "r"(count));
+}
+__device__ __forceinline__ void bar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(saddr(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(saddr(bar)) : "memory");
+}
+__device__ __forceinline__ bool bar_try(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(saddr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  `dead` latches for the calling thread once any wait in the CTA has run out.
+__device__ __forceinline__ void bar_wait(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag)
+{
+    if (dead) return;
+    for (uint32_t i = 0; i < kSpin; ++i) {
+        if (bar_try(bar, parity)) return;
+        if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
+    }
+    dead = true;
+    atomicExch(abort_flag, 1);
 }
 
-int launch_score_tc(const pkv_shape *, const void *, pkv_strides, const void *, pkv_strides,
-                    const float *, const float *, float *, void *, cudaStream_t)
+__device__ __forceinline__ void tma_load_5d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1,
+                                            int c2, int c3, int c4)
 {
-    return PKV_ERR_UNSUPPORTED;
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(saddr(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(saddr(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor, K-major operand with the 128-byte swizzle: rows of 128 bytes,
+// eight-row groups 1024 bytes apart, tile base aligned to 1024 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFFu) >> 4);  // start address, bits [0,14)
+    d |= (uint64_t)1 << 16;                   // leading byte offset (not used by swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;         // stride byte offset, bits [32,46)
+    d |= (uint64_t)1 << 46;                   // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;                   // layout type: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = N = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TT >> 3) << 17) |
+                            ((uint32_t)(TT >> 4) << 24);
+
+__device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(saddr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+
+struct Ring2 {
+    int idx;
+    uint32_t phase;
+    __device__ __forceinline__ void next(int n)
+    {
+        if (++idx == n) {
+            idx = 0;
+            phase ^= 1u;
+        }
+    }
+};
+
+// Work item w -> (segment-head sh, tile t).  Items with the most inner tiles come first.
+template <int PASS> __device__ __forceinline__ void decode_item(int w, int nsh, int tiles, int &sh, int &t)
+{
+    const int rank = w / nsh;
+    sh = w - rank * nsh;
+    t = PASS == 1 ? tiles - 1 - rank : rank;
+}
+
+// PASS 1: stationary = Q tile t, streamed = K tiles 0..t.  PASS 2: stationary = K tile t,
+// streamed = Q tiles t..tiles-1.
+template <int PASS, int D>
+__global__ void __launch_bounds__(192, 2)
+score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                  const ScoreArgs a)
+{
+    constexpr int KH = D / 64;                  // 128-byte swizzle atoms along the head dimension
+    constexpr uint32_t HALF = TT * 128;         // bytes of one [128 rows x 64 elements] box
+    constexpr uint32_t TILE = KH * HALF;        // bytes of one operand tile
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *base = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sA = base;
+    unsigned char *sB = base + TILE;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sB + kStagesB * TILE);
+    uint64_t *a_full = bars, *a_empty = bars + 1, *b_full = bars + 2, *b_empty = b_full + kStagesB;
+    uint64_t *s_full = b_empty + kStagesB, *s_empty = s_full + 2;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s_empty + 2);
+    __shared__ int s_abort;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const CUtensorMap *map_stat = PASS == 1 ? &map_q : &map_k;
+    const CUtensorMap *map_strm = PASS == 1 ? &map_k : &map_q;
+    const int nsh = a.nseg * a.H;
+    const int nitems = nsh * a.tiles;
+
+    if (tid == 0) {
+        s_abort = 0;
+        bar_init(a_full, 1);
+        bar_init(a_empty, 1);
+        for (int i = 0; i < kStagesB; ++i) {
+            bar_init(b_full + i, 1);
+            bar_init(b_empty + i, 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            bar_init(s_full + i, 1);
+            bar_init(s_empty + i, 4);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {  // two 128-column fp32 accumulators
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(saddr(tmem_slot)),
+                     "r"(256u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---- TMA producer ---------------------------------------------------------------------
+        if (lane == 0) {
+            bool dead = false;
+            uint32_t a_phase = 0;
+            Ring2 rb{0, 0u};
+            for (int w = blockIdx.x; w < nitems && !dead; w += gridDim.x) {
+                int sh, t;
+                decode_item<PASS>(w, nsh, a.tiles, sh, t);
+                const int seg = sh / a.H, h = sh - seg * a.H, b = seg / a.L, l = seg - b * a.L;
+                bar_wait(a_empty, a_phase ^ 1u, dead, &s_abort);
+                if (dead) break;
+                bar_expect_tx(a_full, TILE);
+#pragma unroll
+                for (int kh = 0; kh < KH; ++kh)
+                    tma_load_5d(sA + kh * HALF, map_stat, a_full, kh * 64, t * TT, h, l, b);
+                a_phase ^= 1u;
+                const int j0 = PASS == 1 ? 0 : t, j1 = PASS == 1 ? t : a.tiles - 1;
+                for (int j = j0; j <= j1; ++j) {
+                    bar_wait(b_empty + rb.idx, rb.phase ^ 1u, dead, &s_abort);
+                    if (dead) break;
+                    bar_expect_tx(b_full + rb.idx, TILE);
+#pragma unroll
+                    for (int kh = 0; kh < KH; ++kh)
+                        tma_load_5d(sB + rb.idx * TILE + kh * HALF, map_strm, b_full + rb.idx, kh * 64, j * TT, h, l, b);
+                    rb.next(kStagesB);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer -------------------------------------------------------------------------
+        if (lane == 0) {
+            bool dead = false;
+            uint32_t a_phase = 0;
+            Ring2 rb{0, 0u}, rs{0, 0u};
+            for (int w = blockIdx.x; w < nitems && !dead; w += gridDim.x) {
+                int sh, t;
+                decode_item<PASS>(w, nsh, a.tiles, sh, t);
+                bar_wait(a_full, a_phase, dead, &s_abort);
+                a_phase ^= 1u;
+                const int count = PASS == 1 ? t + 1 : a.tiles - t;
+                for (int jj = 0; jj < count && !dead; ++jj) {
+                    bar_wait(b_full + rb.idx, rb.phase, dead, &s_abort);
+                    bar_wait(s_empty + rs.idx, rs.phase ^ 1u, dead, &s_abort);
+                    if (dead) break;
+                    fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)rs.idx * TT;
+                    const uint32_t a_addr = saddr(sA), b_addr = saddr(sB + rb.idx * TILE);
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t off = (uint32_t)(k / 4) * HALF + (uint32_t)(k % 4) * 32;
+                        mma_bf16(d_tmem, smem_desc(a_addr + off), smem_desc(b_addr + off), k > 0 ? 1u : 0u);
+                    }
+                    mma_commit(b_empty + rb.idx);  // the streamed stage is free once these MMAs retire
+                    mma_commit(s_full + rs.idx);   // and the accumulator is ready to be read
+                    rb.next(kStagesB);
+                    rs.next(2);
+                }
+                if (!dead) mma_commit(a_empty);     // the stationary tile may be replaced
+            }
+        }
+    } else {
+        // ---- accumulator readers: one TMEM lane (tile row) per thread ----------------------------
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        bool dead = false;
+        Ring2 rs{0, 0u};
+        for (int w = blockIdx.x; w < nitems; w += gridDim.x) {
+            int sh, t;
+            decode_item<PASS>(w, nsh, a.tiles, sh, t);
+            const int seg = sh / a.H, l = seg % a.L;
+            const float sc = a.layer_scale[l] * kLog2eT;
+            const int grow = t * TT + row;  // query (pass 1) or key (pass 2) index of this thread
+            const float *lse_row = a.lse2 + (size_t)sh * a.Npad;
+            float run_max = -INFINITY, run_sum = 0.f;  // pass 1
+            float col_sum = 0.f;                       // pass 2
+            const int j0 = PASS == 1 ? 0 : t, j1 = PASS == 1 ? t : a.tiles - 1;
+            for (int j = j0; j <= j1; ++j) {
+                bar_wait(s_full + rs.idx, rs.phase, dead, &s_abort);
+                fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)rs.idx * TT;
+                const bool diag = j == t;
+#pragma unroll 1
+                for (int cblk = 0; cblk < TT / 32; ++cblk) {
+                    float v[32];
+                    tmem_ld32(taddr + cblk * 32, v);
+                    if (PASS == 1) {
+                        float cmax = -INFINITY;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            v[i] = (!diag || cblk * 32 + i <= row) ? v[i] * sc : -INFINITY;
+                            cmax = fmaxf(cmax, v[i]);
+                        }
+                        const float nm = fmaxf(run_max, cmax);
+                        if (nm > -INFINITY) {
+                            float part = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) part += exp2f(v[i] - nm);
+                            run_sum = run_sum * exp2f(run_max - nm) + part;
+                            run_max = nm;
+                        }
+                    } else {
+                        const float4 *lp = reinterpret_cast<const float4 *>(lse_row + j * TT + cblk * 32);
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const float4 ls = __ldg(lp + i4);
+                            const float lv[4] = {ls.x, ls.y, ls.z, ls.w};
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int i = i4 * 4 + u;
+                                const float p = exp2f(fmaf(v[i], sc, -lv[u]));
+                                col_sum += (!diag || cblk * 32 + i >= row) ? p : 0.f;
+                            }
+                        }
+                    }
+                }
+                fence_before();
+                __syncwarp();
+                if (lane == 0) bar_arrive(s_empty + rs.idx);
+                rs.next(2);
+            }
+            if (PASS == 1) {
+                a.lse2[(size_t)sh * a.Npad + grow] = grow < a.N ? run_max + log2f(run_sum) : INFINITY;
+            } else if (grow < a.N) {
+                a.partial[(size_t)sh * a.N + grow] = col_sum;
+            }
+        }
+        if (dead && lane == 0 && a.abort_word) atomicExch(a.abort_word, (int)PKV_DEV_TIMEOUT);
+    }
+
+    fence_before();
+    __syncthreads();
+    fence_after();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    }
+}
+
+// Caller-supplied natural-log lse [B*L*H][N] -> padded log2 layout.
+__global__ void convert_lse_kernel(const float *__restrict__ lse, int N, int Npad, size_t rows,
+                                   float *__restrict__ lse2)
+{
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= rows * Npad) return;
+    size_t r = i / Npad;
+    int n = (int)(i - r * Npad);
+    lse2[i] = n < N ? lse[r * N + n] * kLog2eT : INFINITY;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// [B, L, H, N, D] bf16 with element strides -> rank-5 map, box = 64 elements x 128 rows.
+bool make_map(CUtensorMap *map, const void *ptr, const pkv_shape *s, pkv_strides st)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {(cuuint64_t)s->head_dim, (cuuint64_t)s->prompt_len, (cuuint64_t)s->heads,
+                          (cuuint64_t)s->layers, (cuuint64_t)s->batch};
+    int64_t es[4] = {st.n, st.h, st.l, st.b};
+    cuuint64_t strides[4];
+    for (int i = 0; i < 4; ++i) {
+        int64_t v = es[i];
+        if (dims[i + 1] == 1 && v == 0) v = s->head_dim;  // a size-1 dimension's stride is never used
+        strides[i] = (cuuint64_t)v * 2;
+        if (strides[i] % 16 != 0 || strides[i] >= ((cuuint64_t)1 << 40) || strides[i] == 0) return false;
+    }
+    cuuint32_t box[5] = {64, TT, 1, 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void *>(ptr), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+template <int PASS, int D>
+int launch_pass(const CUtensorMap &mq, const CUtensorMap &mk, const ScoreArgs &a, int sms, cudaStream_t st)
+{
+    static bool done[64] = {};
+    const size_t smem = (size_t)(1 + kStagesB) * (D / 64) * TT * 128 + 1024 + 256;
+    int rc = ensure_dynamic_smem((const void *)score_tile_kernel<PASS, D>, (int)smem, done);
+    if (rc != PKV_OK) return rc;
+    const int items = a.nseg * a.H * a.tiles;
+    const int grid = items < 2 * sms ? items : 2 * sms;
+    score_tile_kernel<PASS, D><<<grid, 192, smem, st>>>(mq, mk, a);
+    return check_launch(PASS == 1 ? "score_tile_kernel<1>" : "score_tile_kernel<2>");
+}
+
+}  // namespace
+
+int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, cudaStream_t st);
+
+bool score_tc_usable(const pkv_shape *s, const void *, pkv_strides, const void *, pkv_strides)
+{
+    return s->dtype == PKV_BF16 && (s->head_dim == 64 || s->head_dim == 128) && encode_fn() != nullptr;
+}
+
+size_t score_tc_ws_bytes(const pkv_shape *s)
+{
+    const size_t rows = (size_t)s->batch * s->layers * s->heads;
+    const size_t npad = ((size_t)s->prompt_len + TT - 1) / TT * TT;
+    return round_up(rows * s->prompt_len * sizeof(float), kWsAlign) + round_up(rows * npad * sizeof(float), kWsAlign);
+}
+
+// Returns PKV_OK, an error, or -1 when the tensor maps cannot describe the caller's layout.
+int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const void *k, pkv_strides ks,
+                    const float *scale, const float *lse, float *scores, void *ws, cudaStream_t st)
+{
+    CUtensorMap mq, mk;
+    if (!make_map(&mq, q, s, qs) || !make_map(&mk, k, s, ks)) return -1;
+    const int B = s->batch, L = s->layers, H = s->heads, N = s->prompt_len;
+    const size_t rows = (size_t)B * L * H;
+    ScoreArgs a;
+    a.layer_scale = scale;
+    a.partial = (float *)ws;
+    a.lse2 = (float *)((unsigned char *)ws + round_up(rows * N * sizeof(float), kWsAlign));
+    a.abort_word = nullptr;
+    a.L = L; a.H = H; a.N = N;
+    a.tiles = (N + TT - 1) / TT;
+    a.Npad = a.tiles * TT;
+    a.nseg = B * L;
+
+    static int sm_count[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 0;
+    if (!sms) {
+        cudaError_t e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "cudaDeviceGetAttribute(sm count)");
+            return PKV_ERR_CUDA;
+        }
+        if (dev >= 0 && dev < 64) sm_count[dev] = sms;
+    }
+    int rc;
+    if (lse) {
+        const size_t n = rows * a.Npad;
+        convert_lse_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(lse, N, a.Npad, rows, a.lse2);
+        rc = check_launch("convert_lse_kernel");
+    } else {
+        rc = s->head_dim == 128 ? launch_pass<1, 128>(mq, mk, a, sms, st) : launch_pass<1, 64>(mq, mk, a, sms, st);
+    }
+    if (rc != PKV_OK) return rc;
+    rc = s->head_dim == 128 ? launch_pass<2, 128>(mq, mk, a, sms, st) : launch_pass<2, 64>(mq, mk, a, sms, st);
+    if (rc != PKV_OK) return rc;
+    return launch_head_mean(a.partial, H, N, (size_t)B * L * N, scores, st);
 }
 
 }  // namespace pkv
