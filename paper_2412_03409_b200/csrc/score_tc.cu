@@ -27,7 +27,8 @@ namespace {
 
 constexpr int TT = 128;            // tile side
 constexpr int kStagesB = 2;        // streamed-operand stages
-constexpr uint32_t kSpin = 1u << 22;
+constexpr uint32_t kSpin = 1u << 20;       // tries per wait; each may sleep up to kSuspendNs
+constexpr uint32_t kSuspendNs = 2000;      // suspend-time hint of one try: a waiting thread leaves the issue slots alone
 constexpr float kLog2eT = 1.4426950408889634f;
 
 struct ScoreArgs {
@@ -58,10 +59,10 @@ __device__ __forceinline__ bool bar_try(uint64_t *bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(saddr(bar)), "r"(parity)
+        : "r"(saddr(bar)), "r"(parity), "r"(kSuspendNs)
         : "memory");
     return ok != 0;
 }
@@ -71,7 +72,7 @@ __device__ __forceinline__ void bar_wait(uint64_t *bar, uint32_t parity, bool &d
     if (dead) return;
     for (uint32_t i = 0; i < kSpin; ++i) {
         if (bar_try(bar, parity)) return;
-        if ((i & 1023u) == 1023u && *(volatile int *)abort_flag) break;
+        if ((i & 255u) == 255u && *(volatile int *)abort_flag) break;
     }
     dead = true;
     atomicExch(abort_flag, 1);
@@ -176,6 +177,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     uint64_t *s_full = b_empty + kStagesB, *s_empty = s_full + 2;
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s_empty + 2);
     __shared__ int s_abort;
+    __shared__ __align__(16) float s_lse[2][TT];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const CUtensorMap *map_stat = PASS == 1 ? &map_q : &map_k;
@@ -273,6 +275,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---- accumulator readers: one TMEM lane (tile row) per thread ----------------------------
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
+        const int rtid = tid - 64;  // 0..127 among the reader warps
         bool dead = false;
         Ring2 rs{0, 0u};
         for (int w = blockIdx.x; w < nitems; w += gridDim.x) {
@@ -280,48 +283,74 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             decode_item<PASS>(w, nsh, a.tiles, sh, t);
             const int seg = sh / a.H, l = seg % a.L;
             const float sc = a.layer_scale[l] * kLog2eT;
+            const bool fast = sc > 0.f;     // the usual case: the extreme of sc * x is sc * max x
             const int grow = t * TT + row;  // query (pass 1) or key (pass 2) index of this thread
             const float *lse_row = a.lse2 + (size_t)sh * a.Npad;
             float run_max = -INFINITY, run_sum = 0.f;  // pass 1
             float col_sum = 0.f;                       // pass 2
             const int j0 = PASS == 1 ? 0 : t, j1 = PASS == 1 ? t : a.tiles - 1;
             for (int j = j0; j <= j1; ++j) {
+                if (PASS == 2) {  // this tile's 128 query normalisers, shared by all readers
+                    s_lse[rs.idx][rtid] = __ldg(lse_row + j * TT + rtid);
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
                 bar_wait(s_full + rs.idx, rs.phase, dead, &s_abort);
                 fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)rs.idx * TT;
                 const bool diag = j == t;
+                // On the diagonal tile only the 32-column blocks that reach this warp's rows matter:
+                // blocks 0..quarter in pass 1 (keys <= query), quarter..3 in pass 2 (queries >= key).
+                const int c_lo = (PASS == 2 && diag) ? quarter : 0;
+                const int c_hi = (PASS == 1 && diag) ? quarter : TT / 32 - 1;
 #pragma unroll 1
-                for (int cblk = 0; cblk < TT / 32; ++cblk) {
+                for (int cblk = c_lo; cblk <= c_hi; ++cblk) {
                     float v[32];
                     tmem_ld32(taddr + cblk * 32, v);
+                    const bool edge = diag && cblk == quarter;  // the block the causal boundary crosses
                     if (PASS == 1) {
-                        float cmax = -INFINITY;
+                        if (edge) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            v[i] = (!diag || cblk * 32 + i <= row) ? v[i] * sc : -INFINITY;
-                            cmax = fmaxf(cmax, v[i]);
+                            for (int i = 0; i < 32; ++i) v[i] = i <= lane ? v[i] : -INFINITY;
                         }
-                        const float nm = fmaxf(run_max, cmax);
-                        if (nm > -INFINITY) {
+                        if (fast) {
+                            float cmax = v[0];
+#pragma unroll
+                            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
+                            const float nm = fmaxf(run_max, cmax * sc);  // finite: column 0 is never masked
+                            float part = 0.f;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) part += exp2f(fmaf(v[i], sc, -nm));
+                            run_sum = fmaf(run_sum, exp2f(run_max - nm), part);
+                            run_max = nm;
+                        } else {
+                            float cmax = -INFINITY;
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                v[i] = v[i] == -INFINITY ? -INFINITY : v[i] * sc;
+                                cmax = fmaxf(cmax, v[i]);
+                            }
+                            const float nm = fmaxf(run_max, cmax);
                             float part = 0.f;
 #pragma unroll
                             for (int i = 0; i < 32; ++i) part += exp2f(v[i] - nm);
-                            run_sum = run_sum * exp2f(run_max - nm) + part;
+                            run_sum = fmaf(run_sum, exp2f(run_max - nm), part);
                             run_max = nm;
                         }
                     } else {
-                        const float4 *lp = reinterpret_cast<const float4 *>(lse_row + j * TT + cblk * 32);
+                        const float4 *lp = reinterpret_cast<const float4 *>(&s_lse[rs.idx][cblk * 32]);
+                        float part = 0.f;
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
-                            const float4 ls = __ldg(lp + i4);
+                            const float4 ls = lp[i4];
                             const float lv[4] = {ls.x, ls.y, ls.z, ls.w};
 #pragma unroll
                             for (int u = 0; u < 4; ++u) {
                                 const int i = i4 * 4 + u;
                                 const float p = exp2f(fmaf(v[i], sc, -lv[u]));
-                                col_sum += (!diag || cblk * 32 + i >= row) ? p : 0.f;
+                                part += (!edge || i >= lane) ? p : 0.f;
                             }
                         }
+                        col_sum += part;
                     }
                 }
                 fence_before();
