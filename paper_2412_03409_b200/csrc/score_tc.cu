@@ -135,6 +135,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+// 2^x on the special-function unit, one instruction (inputs here are <= 0 or -inf; flushing
+// denormal results to zero is harmless for sums of probabilities).
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 
@@ -150,12 +158,16 @@ struct Ring2 {
     }
 };
 
-// Work item w -> (segment-head sh, tile t).  Items with the most inner tiles come first.
+// Work item w -> (segment-head sh, tile t).  The tiles of one head are consecutive items, so
+// the CTAs running at any moment share a few dozen heads whose Q and K stay in L2 and every
+// operand byte comes from HBM once per pass.  Pass 2 walks the heads backwards: it starts on
+// what pass 1 touched last.  A CTA's successive items (stride gridDim.x) cycle through the
+// tile index, which mixes long and short items evenly.
 template <int PASS> __device__ __forceinline__ void decode_item(int w, int nsh, int tiles, int &sh, int &t)
 {
-    const int rank = w / nsh;
-    sh = w - rank * nsh;
-    t = PASS == 1 ? tiles - 1 - rank : rank;
+    const int q = w / tiles;
+    t = w - q * tiles;
+    sh = PASS == 1 ? q : nsh - 1 - q;
 }
 
 // PASS 1: stationary = Q tile t, streamed = K tiles 0..t.  PASS 2: stationary = K tile t,
@@ -319,8 +331,8 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             const float nm = fmaxf(run_max, cmax * sc);  // finite: column 0 is never masked
                             float part = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) part += exp2f(fmaf(v[i], sc, -nm));
-                            run_sum = fmaf(run_sum, exp2f(run_max - nm), part);
+                            for (int i = 0; i < 32; ++i) part += ex2(fmaf(v[i], sc, -nm));
+                            run_sum = fmaf(run_sum, ex2(run_max - nm), part);
                             run_max = nm;
                         } else {
                             float cmax = -INFINITY;
@@ -332,8 +344,8 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             const float nm = fmaxf(run_max, cmax);
                             float part = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) part += exp2f(v[i] - nm);
-                            run_sum = fmaf(run_sum, exp2f(run_max - nm), part);
+                            for (int i = 0; i < 32; ++i) part += ex2(v[i] - nm);
+                            run_sum = fmaf(run_sum, ex2(run_max - nm), part);
                             run_max = nm;
                         }
                     } else {
@@ -346,7 +358,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                             for (int u = 0; u < 4; ++u) {
                                 const int i = i4 * 4 + u;
-                                const float p = exp2f(fmaf(v[i], sc, -lv[u]));
+                                const float p = ex2(fmaf(v[i], sc, -lv[u]));
                                 part += (!edge || i >= lane) ? p : 0.f;
                             }
                         }
