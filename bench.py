@@ -183,7 +183,7 @@ def run_ours(args):
     import torch
     import torch.distributed as dist
 
-    from paper_2412_03409_b200 import api, workloads as wl
+    from paper_2412_03409_b200 import api, sharding, workloads as wl
     from paper_2412_03409_b200.session import Session
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -204,8 +204,7 @@ def run_ours(args):
     R = max(1, min(8, 1 + -(-(256 << 20) // retained_bytes))) if retained_bytes < (256 << 20) else 1
     # Ranks hold different samples of the same workload (batch sharding, no exchange).
     reps = []
-    for r in range(R):
-        samples = [(rank * R + r) * w.B + b for b in range(w.B)]
+    for samples in sharding.samples_for_rank(rank, world, w.B, R):
         q, k, v = wl.make_prompt(w, dev, samples=samples)
         s = Session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T, max_budget_rows=budget,
                     device=dev)
@@ -265,10 +264,7 @@ def run_ours(args):
     for kx in stage_ms:
         stage_ms[kx] /= args.steps * R
     step_ms = sum(stage_ms.values())
-    t_max = torch.tensor([step_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    step_ms_max = float(t_max.item())
+    step_ms_max = sharding.max_over_ranks(step_ms, dev)
 
     # algorithmic bytes of the decode steps (rows actually attended, K and V, plus the append)
     lens = (s.cache.len.cpu().to(torch.int64) - w.T)      # retained rows after compaction
@@ -287,10 +283,7 @@ def run_ours(args):
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, max(2, min(args.steps, 5)))
-        if world > 1:
-            t = torch.tensor([e2e["ms"]], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e["ms"] = float(t.item())
+        e2e["ms"] = sharding.max_over_ranks(e2e["ms"], dev)
 
     if rank != 0:
         if world > 1:

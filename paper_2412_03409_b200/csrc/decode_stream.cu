@@ -35,9 +35,9 @@ struct DecodeArgs {
     const int32_t *cap;
     const float *layer_scale;
     float *scratch;   // partial slots
+    int *plan;        // [nact] int4 records written by the stream kernel for the merge kernel
     int32_t *dev_status;
     int L, H, layer_begin, nl, nact, nseg_total, nstages, nwarps;
-    int unit_rows, grid;  // rows per unit and CTAs of the stream kernel (the merge kernel re-derives its plan)
     uint32_t row_bytes;
     int64_t total_cap_rows;
 };
@@ -251,6 +251,19 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
     const int upc = G > 0 ? U / G : 0, rem = G > 0 ? U - upc * G : 0;
     // The merge kernel may be scheduled from here on; it still waits for this grid to finish.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (cta == 0) {
+        // The plan, for the merge kernel: rows, first contributing CTA and number of contributing
+        // CTAs of every active segment.  (That kernel must not rebuild it from len, which it bumps.)
+        for (int i = tid; i < a.nact; i += blockDim.x) {
+            const int rows = seg_n[i];
+            int first = 0, cnt = 0;
+            if (rows >= 0) {
+                first = unit_owner(P[i], upc, rem);
+                cnt = unit_owner(P[i + 1] - 1, upc, rem) - first + 1;
+            }
+            reinterpret_cast<int4 *>(a.plan)[i] = make_int4(rows, first, cnt, 0);
+        }
+    }
     if (cta < G) {
         u0 = first_unit(cta, upc, rem);
         u1 = first_unit(cta + 1, upc, rem);
@@ -533,10 +546,10 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 }
 
 // Merge kernel: one warp per (head, active segment), launched as a programmatic dependent of
-// the stream kernel.  Before it waits for that grid it rebuilds the unit plan from the
-// lengths (which the stream kernel only reads), so that afterwards one round trip fetches
-// the partials of up to 16 contributing CTAs at once.  For a segment split over several CTAs
-// it combines their partials; for every segment that took a row, the warp of head 0 bumps len.
+// the stream kernel, whose CTA 0 leaves it one record per segment (rows, first contributing CTA,
+// number of contributors).  For a segment split over several CTAs it combines their partials,
+// up to 16 contributors per round trip; for every segment that took a row, the warp of head 0
+// bumps len.  It reads len nowhere: blocks of a large grid start after others have bumped it.
 template <typename T, int D>
 __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
 {
@@ -544,39 +557,10 @@ __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
     constexpr int KB = 16;  // contributors per batch
     const int h = blockIdx.x, si = blockIdx.y, lane = threadIdx.x;
 
-    // ---- same plan as the stream kernel: units before this segment, in it, and in total ------
-    int before = 0, mine = 0, total = 0, n = -1;
-    for (int base = 0; base < a.nact; base += 32) {
-        const int i = base + lane;
-        int units = 0;
-        if (i < a.nact) {
-            const int rows = segment_rows(a, i);
-            units = rows >= 0 ? (rows + a.unit_rows) / a.unit_rows : 0;
-            if (i == si) n = rows;
-        }
-        int incl = units;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        if (si >= base && si < base + 32) {
-            before = total + __shfl_sync(0xffffffffu, incl - units, si - base);
-            mine = __shfl_sync(0xffffffffu, units, si - base);
-        }
-        total += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    n = __shfl_sync(0xffffffffu, n, si & 31);
-    const int G = a.grid < total ? a.grid : total;
-    const int upc = G > 0 ? total / G : 0, rem = G > 0 ? total - upc * G : 0;
     const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-    int c_first = 0, ncontrib = 0;
-    if (n >= 0) {
-        c_first = unit_owner(before, upc, rem);
-        ncontrib = unit_owner(before + mine - 1, upc, rem) - c_first + 1;
-    }
-
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
+    const int4 rec = reinterpret_cast<const int4 *>(a.plan)[si];
+    const int n = rec.x, c_first = rec.y, ncontrib = rec.z;
     if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
     if (h == 0 && lane == 0) a.len[seg] = n + 1;
     if (ncontrib == 1) return;
@@ -620,11 +604,14 @@ __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
     for (int i = 0; i < D / 32; ++i) dst[lane + 32 * i] = from_float<T>(o[i] * inv);
 }
 
+static size_t plan_bytes(int nact) { return round_up((size_t)nact * sizeof(int4), kWsAlign); }
+
 size_t decode_stream_ws_bytes(const pkv_shape *s)
 {
     size_t nseg = (size_t)s->batch * s->layers;
     size_t slots = 256 + nseg;
-    return round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
+    return plan_bytes((int)(nseg < (size_t)kMaxActive ? nseg : kMaxActive)) +
+           round_up(slots * s->heads * (s->head_dim + 4) * sizeof(float), kWsAlign);
 }
 
 static size_t stream_smem_bytes(int nstages, int ur, uint32_t rb, int nact)
@@ -702,12 +689,11 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     a.q = q; a.k_new = kn; a.v_new = vn; a.ck = c->k; a.cv = c->v; a.out = out;
     a.row_offset = c->row_offset; a.len = c->len; a.cap = c->cap;
     a.layer_scale = scale; a.dev_status = dev_status;
-    a.scratch = (float *)ws;
+    a.plan = (int *)ws;
+    a.scratch = (float *)((unsigned char *)ws + plan_bytes(nact));
     a.L = s->layers; a.H = H; a.layer_begin = lb; a.nl = nl; a.nact = nact;
     a.nseg_total = s->batch * s->layers; a.nstages = nstages; a.row_bytes = row_bytes;
     a.total_cap_rows = c->total_cap_rows;
-    a.unit_rows = ur;
-    a.grid = sms;
 
     const bool bf = s->dtype == PKV_BF16;
     const int vec_per_head = D / (int)(16 / es);

@@ -206,6 +206,7 @@ def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
             cv = np.concatenate([cv, to_np32(vn[b, l])[None]])
             caches[(b, l)] = [ck, cv]
             ref = oracle.decode_attn(to_np32(qd[b, l]), ck, cv, float(layer_scale[l]))
+            assert np.isfinite(got[b, l]).all()
             worst = max(worst, float(np.abs(got[b, l] - ref).max()))
     return worst
 
