@@ -211,6 +211,9 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         P[0] = 0;
     }
+    // Launched as a programmatic dependent of whatever precedes it in the stream: everything
+    // above overlapped that kernel's tail; its writes (lengths, cache rows) are visible from here.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int si = tid; si < a.nact; si += blockDim.x) {
         int64_t off;
         const int rows = segment_rows(a, si, &off);
@@ -558,6 +561,7 @@ __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
     const int h = blockIdx.x, si = blockIdx.y, lane = threadIdx.x;
 
     const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // e.g. the next decode step
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
     const int4 rec = reinterpret_cast<const int4 *>(a.plan)[si];
     const int n = rec.x, c_first = rec.y, ncontrib = rec.z;
@@ -627,23 +631,30 @@ static int launch_variant(const DecodeArgs &a, int sms, cudaStream_t st)
     if ((a.nwarps + 1) * 32 > MAXT) return -1;
     int rc = ensure_dynamic_smem((const void *)decode_stream_kernel<T, D, LPR, HPW, UR, MAXT>, kDynSmemMax, done);
     if (rc != PKV_OK) return rc;
-    decode_stream_kernel<T, D, LPR, HPW, UR, MAXT>
-        <<<sms, (a.nwarps + 1) * 32, stream_smem_bytes(a.nstages, UR, a.row_bytes, a.nact), st>>>(a);
-    rc = check_launch("decode_stream_kernel");
-    if (rc != PKV_OK) return rc;
-    // The merge kernel is a programmatic dependent: it may be set up while the stream kernel
-    // runs and starts past its griddepcontrol.wait once that grid has completed.
+    // Both kernels are programmatic dependents of their predecessor in the stream: they may be
+    // set up while it still runs and go past their griddepcontrol.wait once it has completed.
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sms);
+    cfg.blockDim = dim3((a.nwarps + 1) * 32);
+    cfg.dynamicSmemBytes = stream_smem_bytes(a.nstages, UR, a.row_bytes, a.nact);
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_stream_kernel<T, D, LPR, HPW, UR, MAXT>, a);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "decode_stream_kernel");
+        return PKV_ERR_CUDA;
+    }
     cfg.gridDim = dim3(a.H, a.nact);
     cfg.blockDim = dim3(32);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D>, a);
+    e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D>, a);
     if (e != cudaSuccess) {
         set_cuda_error(e, "decode_finish_kernel");
         return PKV_ERR_CUDA;
