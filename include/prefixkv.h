@@ -140,6 +140,32 @@ int prefixkv_apply_lengths(const pkv_shape *shape, const float *scores, const in
                            int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Meeting the budget exactly after an inexact search (Sec. 3.3: "scale the resulting global
+ * prefix configuration to meet the target budget"; the paper prints no formula).  Reading:
+ * every layer keeps its one mandatory row and the other budget - L rows are split in
+ * proportion to len - 1 (largest remainder, ties to the lower layer, at most N rows per
+ * layer).  A configuration that already sums to its budget is left unchanged; otherwise
+ * lengths only grow, so each layer keeps a longer prefix of the same priority sequence.
+ *   len          [B,L] int32, in/out (from prefixkv_search)
+ *   budget_rows  [B] int64
+ * Call it between prefixkv_search and prefixkv_compact.
+ */
+int prefixkv_rescale(const pkv_shape *shape, int32_t *len, const int64_t *budget_rows,
+                     int32_t *dev_status, void *cuda_stream);
+
+/*
+ * Offline configuration (Sec. 3.3, last paragraph: the lengths found on a few sample prompts
+ * are applied to every input; the aggregation is not specified).  Reading: the same
+ * apportionment with weight[l] = sum over the B sample prompts of (len[b][l] - 1).
+ *   len          [B,L] int32: per-sample lengths of B sample prompts (prefixkv_search)
+ *   budget_rows  host value: rows the configuration may keep over all layers
+ *   len_out      [L] int32 out: pass it to prefixkv_apply_lengths with per_sample = 0
+ *   dev_status   [B]; conditions are reported on sample 0
+ */
+int prefixkv_estimate_config(const pkv_shape *shape, const int32_t *len, int64_t budget_rows,
+                             int32_t *len_out, int32_t *dev_status, void *cuda_stream);
+
+/*
  * Ragged per-layer cache (Fig. 2a).  Rows of segment s occupy
  * [row_offset[s], row_offset[s] + cap[s]) of k and v; the first len[s] are
  * valid.  A row is one token's vectors for all heads: [H][D] elements.

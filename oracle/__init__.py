@@ -179,3 +179,22 @@ def select_sample(scores, budget, tol=1e-6, max_iters=64, slack=0):
     if status != OK:
         return order, cum, SearchResult(np.zeros(L, np.int32), 0.0, 0, status)
     return order, cum, search(cum, budget, tol, max_iters, slack)
+
+
+def apportion(weight, budget, N):
+    """Split `budget` rows over layers: one each, the rest in proportion to weight[l]."""
+    weight = np.ascontiguousarray(weight, np.int64)
+    out = np.zeros(weight.shape[0], np.int32)
+    st = _L().orc_apportion(_p(weight, ctypes.c_int64), weight.shape[0], ctypes.c_int64(int(budget)),
+                            int(N), _p(out, ctypes.c_int32))
+    return out, int(st)
+
+
+def rescale(length, budget, N):
+    """Stretch a searched configuration (sum <= budget) to meet the budget exactly."""
+    return apportion(np.asarray(length, np.int64) - 1, budget, N)
+
+
+def estimate_config(lengths, budget, N):
+    """One configuration for all inputs from the per-sample lengths[K, L] of K sample prompts."""
+    return apportion((np.asarray(lengths, np.int64) - 1).sum(axis=0), budget, N)

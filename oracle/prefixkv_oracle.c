@@ -289,3 +289,66 @@ double orc_gini(const float *I, const int32_t *order, int N)
     }
     return 1.0 - 2.0 * area;
 }
+
+/* ------------------------------------------------------------------------
+ * Meeting the budget exactly after an inexact search (Sec. 3.3: "scale the
+ * resulting global prefix configuration to meet the target budget"; the paper
+ * gives no formula) and deriving one configuration from several samples
+ * (Sec. 3.3, last paragraph; the aggregation is not specified either).
+ * Reading used for both: every layer keeps its one mandatory row; the other
+ * budget - L rows are split in proportion to weight[l] (largest-remainder
+ * apportionment, ties to the lower layer, at most N rows per layer).
+ *   rescale:  weight[l] = len[l] - 1 of the searched configuration
+ *   estimate: weight[l] = sum over samples of (len[b][l] - 1)
+ * If the searched configuration already sums to the budget it is returned
+ * unchanged.  All arithmetic is integer.
+ * ---------------------------------------------------------------------- */
+int orc_apportion(const int64_t *weight, int L, int64_t budget, int N, int32_t *len_out)
+{
+    if (budget < (int64_t)L) return ORC_BUDGET_TOO_SMALL;
+    int64_t extra = budget - L, cap = (int64_t)N - 1, W = 0;
+    for (int l = 0; l < L; ++l) {
+        if (weight[l] < 0) return ORC_BAD_LENGTH;
+        W += weight[l];
+    }
+    int64_t *w = (int64_t *)malloc((size_t)L * sizeof(int64_t));
+    int64_t *x = (int64_t *)malloc((size_t)L * sizeof(int64_t));
+    int64_t *fr = (int64_t *)malloc((size_t)L * sizeof(int64_t));
+    int *ord = (int *)malloc((size_t)L * sizeof(int));
+    for (int l = 0; l < L; ++l) w[l] = W == 0 ? 1 : weight[l];
+    if (W == 0) W = L;
+    int64_t rem = extra;
+    for (int l = 0; l < L; ++l) {
+        /* w * extra < 2^63 for every supported size (w <= 2^30 rows, extra <= 2^24 rows) */
+        int64_t prod = w[l] * extra;
+        x[l] = prod / W;
+        fr[l] = prod % W;
+        if (x[l] > cap) x[l] = cap;
+        rem -= x[l];
+        ord[l] = l;
+    }
+    /* order: remainder descending, layer ascending (insertion sort, stable) */
+    for (int i = 1; i < L; ++i) {
+        int cur = ord[i], j = i;
+        while (j > 0 && fr[ord[j - 1]] < fr[cur]) {
+            ord[j] = ord[j - 1];
+            --j;
+        }
+        ord[j] = cur;
+    }
+    while (rem > 0) {
+        int given = 0;
+        for (int i = 0; i < L && rem > 0; ++i) {
+            int l = ord[i];
+            if (x[l] < cap) {
+                ++x[l];
+                --rem;
+                ++given;
+            }
+        }
+        if (!given) break; /* every layer already keeps all N rows */
+    }
+    for (int l = 0; l < L; ++l) len_out[l] = (int32_t)(1 + x[l]);
+    free(w); free(x); free(fr); free(ord);
+    return ORC_OK;
+}

@@ -23,7 +23,8 @@ F32, BF16 = 0, 1
 
 EXPORTS = ["prefixkv_workspace_bytes", "prefixkv_last_cuda_error", "prefixkv_score",
            "prefixkv_search", "prefixkv_apply_lengths", "prefixkv_compact",
-           "prefixkv_decode_attn", "prefixkv_gini", "prefixkv_decode_attn_static",
+           "prefixkv_decode_attn", "prefixkv_gini", "prefixkv_rescale",
+           "prefixkv_estimate_config", "prefixkv_decode_attn_static",
            "prefixkv_decode_static_limit_bytes"]
 
 
@@ -69,6 +70,8 @@ def _load():
     lib.prefixkv_decode_attn.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp, i32, i32,
                                          vp, vp, vp, sz, vp]
     lib.prefixkv_gini.argtypes = [sp, vp, vp, vp]
+    lib.prefixkv_rescale.argtypes = [sp, vp, vp, vp, vp]
+    lib.prefixkv_estimate_config.argtypes = [sp, vp, i64, vp, vp, vp]
     lib.prefixkv_decode_attn_static.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp,
                                                 i32, i32, vp, vp, vp]
     for name in EXPORTS[2:-1]:
@@ -217,3 +220,14 @@ def prefixkv_decode_attn_static(shape, cache: Cache, q, k_new, v_new, layer_scal
                                             _ptr(k_new), _ptr(v_new), _ptr(layer_scale),
                                             int(layer_begin), int(le), _ptr(out), _ptr(dev_status),
                                             _stream()), "prefixkv_decode_attn_static")
+
+
+def prefixkv_rescale(shape, length, budget_rows, dev_status):
+    _check(_lib.prefixkv_rescale(ctypes.byref(shape), _ptr(length), _ptr(budget_rows), _ptr(dev_status),
+                                 _stream()), "prefixkv_rescale")
+
+
+def prefixkv_estimate_config(shape, length, budget_rows, len_out, dev_status):
+    _check(_lib.prefixkv_estimate_config(ctypes.byref(shape), _ptr(length), int(budget_rows),
+                                         _ptr(len_out), _ptr(dev_status), _stream()),
+           "prefixkv_estimate_config")

@@ -373,3 +373,40 @@ def test_argument_validation_fails_on_the_host(api):
     with pytest.raises(api.PrefixKVError):                      # workspace too small
         api.prefixkv_decode_attn(s.shape, s.cache, s.out, s.out, s.out, s.layer_scale, s.out,
                                  s.status, torch.empty(256, dtype=torch.uint8, device="cuda"))
+
+
+# --------------------------------------------------------------------------
+# exact budget after an inexact search; offline configuration from sample prompts
+# --------------------------------------------------------------------------
+def test_rescale_and_offline_configuration(api):
+    B, L, N = 6, 32, 640
+    scores = np.stack([wl.synthetic_scores(L, N, seed=b + 300) for b in range(B)])
+    budgets = [L * N // 5 + 7 * b for b in range(B)]
+    s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    # a coarse search (5 midpoints) leaves part of the budget unused
+    s.search(torch.tensor(budgets), tol=0.0, max_iters=5, scores=torch.from_numpy(scores).cuda())
+    searched = s.len.cpu().numpy().copy()
+    assert (searched.sum(axis=1) < np.array(budgets)).any()
+    api.prefixkv_rescale(s.shape, s.len, s.budget, s.status)
+    got = s.len.cpu().numpy()
+    for b in range(B):
+        ref, st = oracle.rescale(searched[b], budgets[b], N)
+        assert st == oracle.OK
+        np.testing.assert_array_equal(got[b], ref)
+        assert got[b].sum() == budgets[b] and (got[b] >= searched[b]).all()
+    assert s.status.cpu().tolist() == [0] * B
+    # one configuration for all inputs from the B sample prompts
+    s.search(torch.tensor(budgets), scores=torch.from_numpy(scores).cuda())
+    per_sample = s.len.cpu().numpy().copy()
+    cfg = torch.zeros(L, dtype=torch.int32, device="cuda")
+    api.prefixkv_estimate_config(s.shape, s.len, budgets[0], cfg, s.status)
+    ref, st = oracle.estimate_config(per_sample, budgets[0], N)
+    assert st == oracle.OK
+    np.testing.assert_array_equal(cfg.cpu().numpy(), ref)
+    assert int(cfg.sum()) == budgets[0]
+    # and it feeds the given-lengths entry point
+    s.apply_lengths(cfg.cpu(), scores=torch.from_numpy(scores).cuda())
+    assert (s.len.cpu().numpy() == ref[None]).all() and s.status.cpu().tolist() == [0] * B
+    # too small a budget is reported
+    api.prefixkv_estimate_config(s.shape, s.len, L - 1, cfg, s.status)
+    assert s.status[0].item() == api.DEV_BUDGET_TOO_SMALL

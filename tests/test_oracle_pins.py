@@ -400,3 +400,69 @@ def test_gini_closed_forms():
     x = np.sort(ramp.astype(np.float64))
     ref = (2 * np.sum(np.arange(1, N + 1) * x) / (N * x.sum())) - (N + 1) / N
     assert abs(g - ref) < 1e-12
+
+
+# --------------------------------------------------------------------------
+# Meeting the budget exactly / offline configuration (Sec. 3.3)
+# --------------------------------------------------------------------------
+def _hamilton(weight, budget, N):
+    """Largest-remainder apportionment with exact rationals (independent of the oracle)."""
+    L = len(weight)
+    extra, cap = budget - L, N - 1
+    w = [int(x) for x in weight]
+    if sum(w) == 0:
+        w = [1] * L
+    W = sum(w)
+    quota = [Fraction(x * extra, W) for x in w]
+    x = [min(cap, q.numerator // q.denominator) for q in quota]
+    order = sorted(range(L), key=lambda l: (-(quota[l] - (quota[l].numerator // quota[l].denominator)), l))
+    rem = extra - sum(x)
+    while rem > 0:
+        given = 0
+        for l in order:
+            if rem > 0 and x[l] < cap:
+                x[l] += 1; rem -= 1; given += 1
+        if not given:
+            break
+    return [1 + v for v in x]
+
+
+def test_rescale_meets_budget_and_keeps_proportions():
+    rng = np.random.default_rng(21)
+    for _ in range(40):
+        L, N = int(rng.integers(1, 12)), int(rng.integers(2, 60))
+        length = rng.integers(1, N + 1, L)
+        budget = int(rng.integers(length.sum(), L * N + 5))
+        out, st = oracle.rescale(length, budget, N)
+        assert st == oracle.OK
+        assert out.sum() == min(budget, L * N)
+        assert (out >= length).all() and (out <= N).all() and (out >= 1).all()
+        assert list(out) == _hamilton(length - 1, budget, N)
+        same, _ = oracle.rescale(length, int(length.sum()), N)      # nothing to do: unchanged
+        np.testing.assert_array_equal(same, length)
+    # the hand-worked search example: budget 4 was missed by one row (len = (1, 2)); the row
+    # goes to the layer with the larger share beyond its mandatory row
+    out, _ = oracle.rescale([1, 2], 4, 3)
+    assert list(out) == [1, 3]
+    assert oracle.rescale([1, 2], 1, 3)[1] == oracle.BUDGET_TOO_SMALL
+
+
+def test_offline_configuration_from_samples():
+    rng = np.random.default_rng(22)
+    K, L, N = 10, 6, 50
+    base = rng.integers(2, N, L)
+    lens = np.clip(base[None] + rng.integers(-2, 3, (K, L)), 1, N)
+    budget = L * N // 3
+    cfg, st = oracle.estimate_config(lens, budget, N)
+    assert st == oracle.OK and cfg.sum() == budget and (cfg >= 1).all() and (cfg <= N).all()
+    assert list(cfg) == _hamilton((lens - 1).sum(axis=0), budget, N)
+    # identical samples: the configuration is the rescaled single-sample one
+    one, _ = oracle.rescale(lens[0], budget, N) if lens[0].sum() <= budget else (None, None)
+    rep, _ = oracle.estimate_config(np.tile(lens[0], (K, 1)), budget, N)
+    assert list(rep) == _hamilton(lens[0] - 1, budget, N)
+    # layers that keep more rows in the samples keep more rows in the configuration
+    order = np.argsort((lens - 1).sum(axis=0))
+    assert (np.diff(cfg[order]) >= 0).all()
+    # all samples at one row per layer: the budget is spread evenly
+    flat, _ = oracle.estimate_config(np.ones((3, 4), np.int64), 10, 20)
+    assert sorted(flat.tolist()) == [2, 2, 3, 3] and flat.sum() == 10
