@@ -198,3 +198,14 @@ def rescale(length, budget, N):
 def estimate_config(lengths, budget, N):
     """One configuration for all inputs from the per-sample lengths[K, L] of K sample prompts."""
     return apportion((np.asarray(lengths, np.int64) - 1).sum(axis=0), budget, N)
+
+
+def decode_slot(len0, N, g, n, d, ring):
+    """Where generated token g goes in a layer's cache (see orc_decode_slot).
+    ring: int32 array of d + 1 entries, updated in place.  Returns (dst, evicted, rows_after)."""
+    assert ring.dtype == np.int32 and ring.flags["C_CONTIGUOUS"] and ring.shape[0] == d + 1
+    dst, ev = ctypes.c_int32(0), ctypes.c_int32(0)
+    _L().orc_decode_slot.restype = ctypes.c_int32
+    rows = _L().orc_decode_slot(int(len0), int(N), int(g), int(n), int(d), _p(ring, ctypes.c_int32),
+                                ctypes.byref(dst), ctypes.byref(ev))
+    return dst.value, bool(ev.value), int(rows)

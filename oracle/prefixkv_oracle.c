@@ -352,3 +352,36 @@ int orc_apportion(const int64_t *weight, int L, int64_t budget, int N, int32_t *
     free(w); free(x); free(fr); free(ord);
     return ORC_OK;
 }
+
+/* ------------------------------------------------------------------------
+ * Keeping the configuration while decoding (Sec. 3.1: "prune the vectors at a
+ * fixed distance to the latest generated token and maintain the global prefix
+ * configuration"; Fig. 2a: the cache "consistently maintains the derived
+ * compression proportions").  The distance and the exact rule are left to the
+ * cited work; reading used here, per layer:
+ *   R_l = len0 / N is the layer's proportion.  When generated token g arrives
+ *   (g = 0, 1, ...) the layer may hold floor(len0 * (N + g + 1) / N) rows.  If
+ *   adding the token would exceed that, the token generated d steps earlier
+ *   (g - d) is dropped -- if it is still cached -- and the new row takes its
+ *   slot; otherwise the new row is appended.  Prompt rows are never dropped.
+ * ring[d + 1] holds the row index of each of the last d + 1 generated tokens
+ * (-1 once dropped), indexed by token % (d + 1).  n = rows cached now.
+ * Outputs: *dst = row the new token is written to, *evict = 1 if it replaced
+ * token g - d; returns the row count afterwards.  d = 0 never drops anything.
+ * ---------------------------------------------------------------------- */
+int32_t orc_decode_slot(int32_t len0, int32_t N, int32_t g, int32_t n, int32_t d, int32_t *ring,
+                        int32_t *dst, int32_t *evict)
+{
+    *evict = 0;
+    *dst = n;
+    if (d > 0) {
+        int64_t target = ((int64_t)len0 * ((int64_t)N + g + 1)) / N;
+        if ((int64_t)n + 1 > target && g >= d && ring[(g - d) % (d + 1)] >= 0) {
+            *evict = 1;
+            *dst = ring[(g - d) % (d + 1)];
+            ring[(g - d) % (d + 1)] = -1;
+        }
+        ring[g % (d + 1)] = *dst;
+    }
+    return *evict ? n : n + 1;
+}

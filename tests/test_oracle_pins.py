@@ -466,3 +466,48 @@ def test_offline_configuration_from_samples():
     # all samples at one row per layer: the budget is spread evenly
     flat, _ = oracle.estimate_config(np.ones((3, 4), np.int64), 10, 20)
     assert sorted(flat.tolist()) == [2, 2, 3, 3] and flat.sum() == 10
+
+
+# --------------------------------------------------------------------------
+# Keeping the proportions while decoding (Sec. 3.1, Fig. 2a)
+# --------------------------------------------------------------------------
+def _token_list_model(len0, N, d, steps):
+    """Independent model: the cache as a list of tokens ('p', i) / ('g', i)."""
+    cache = [("p", i) for i in range(len0)]
+    sizes = []
+    for g in range(steps):
+        target = (len0 * (N + g + 1)) // N
+        victim = ("g", g - d)
+        if d > 0 and len(cache) + 1 > target and g >= d and victim in cache:
+            cache[cache.index(victim)] = ("g", g)          # the new row takes the dropped row's slot
+        else:
+            cache.append(("g", g))
+        sizes.append(len(cache))
+    return cache, sizes
+
+
+@pytest.mark.parametrize("len0,N,d", [(13, 64, 4), (50, 64, 3), (1, 40, 1), (64, 64, 5), (20, 100, 8), (7, 64, 0)])
+def test_decode_time_pruning_rule(len0, N, d):
+    steps = 120
+    ring = np.full(d + 1, -1, np.int32)
+    rows = [("p", i) for i in range(len0)]
+    n = len0
+    for g in range(steps):
+        dst, ev, n_after = oracle.decode_slot(len0, N, g, n, d, ring)
+        if ev:
+            assert rows[dst] == ("g", g - d) and n_after == n
+            rows[dst] = ("g", g)
+        else:
+            assert dst == n and n_after == n + 1
+            rows.append(("g", g))
+        n = n_after
+        # proportion kept: never more than the layer's share plus the d tokens not yet prunable
+        assert d == 0 or n <= (len0 * (N + g + 1)) // N + d
+        assert all(("g", i) in rows for i in range(max(0, g - d + 1), g + 1)) or d == 0   # recent window
+        assert all(("p", i) in rows for i in range(len0))                                  # prompt rows stay
+    ref_rows, ref_sizes = _token_list_model(len0, N, d, steps)
+    assert rows == ref_rows and n == ref_sizes[-1]
+    if d == 0 or len0 == N:
+        assert n == len0 + steps                                                            # nothing dropped
+    else:
+        assert n < len0 + steps
