@@ -178,6 +178,12 @@ typedef struct {
     int32_t *cap;           /* [B*L] out: len after compaction + decode_cap              */
     int64_t total_cap_rows; /* host: rows allocated; must cover sum(len) + B*L*decode_cap */
     int32_t decode_cap;     /* host: rows of head-room per segment for decoding          */
+    /* Decode-time pruning (optional; evict_distance = 0 or NULL pointers: the cache only grows). */
+    int32_t evict_distance; /* host: d > 0 drops the token generated d steps ago when a layer
+                               would exceed its proportion len0 / N of the sequence            */
+    int32_t *len0;          /* [B*L] out: rows kept by compaction                              */
+    int32_t *gen;           /* [B*L] out: tokens decoded so far                                */
+    int32_t *slot_ring;     /* [B*L][evict_distance + 1] out: row of each recent token, -1 once dropped */
 } pkv_cache;
 
 /*
@@ -204,7 +210,12 @@ int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, cons
  * over all len + 1 rows, and set len += 1.
  *   q, k_new, v_new, out   [B,L,H,D] contiguous, dtype of the cache
  * A segment already at capacity raises PKV_DEV_CAPACITY, appends nothing and
- * writes zeros.  Calls on one cache, or sharing one workspace, must not overlap on
+ * writes zeros.
+ * With cache->evict_distance = d > 0 the layer proportions are kept while decoding (Sec. 3.1,
+ * Fig. 2a; the distance and the exact rule are the cited work's, this is the reading): when
+ * generated token g would push a layer past floor(len0 * (N + g + 1) / N) rows and token
+ * g - d is still cached, the new row takes that token's slot and len stays; otherwise it is
+ * appended.  Prompt rows are never dropped.  Calls on one cache, or sharing one workspace, must not overlap on
  * the GPU.
  */
 int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, const void *q,

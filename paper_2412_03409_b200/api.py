@@ -42,7 +42,9 @@ class Strides(ctypes.Structure):
 class CacheStruct(ctypes.Structure):
     _fields_ = [("k", ctypes.c_void_p), ("v", ctypes.c_void_p), ("row_offset", ctypes.c_void_p),
                 ("len", ctypes.c_void_p), ("cap", ctypes.c_void_p),
-                ("total_cap_rows", ctypes.c_int64), ("decode_cap", ctypes.c_int32)]
+                ("total_cap_rows", ctypes.c_int64), ("decode_cap", ctypes.c_int32),
+                ("evict_distance", ctypes.c_int32), ("len0", ctypes.c_void_p),
+                ("gen", ctypes.c_void_p), ("slot_ring", ctypes.c_void_p)]
 
 
 class PrefixKVError(RuntimeError):
@@ -160,15 +162,23 @@ class Cache:
     cap: torch.Tensor
     total_cap_rows: int
     decode_cap: int
+    evict_distance: int = 0
+    len0: torch.Tensor = None
+    gen: torch.Tensor = None
+    slot_ring: torch.Tensor = None
     c: CacheStruct = None
 
     def __post_init__(self):
         self.c = CacheStruct(self.k.data_ptr(), self.v.data_ptr(), self.row_offset.data_ptr(),
                              self.len.data_ptr(), self.cap.data_ptr(), self.total_cap_rows,
-                             self.decode_cap)
+                             self.decode_cap, self.evict_distance,
+                             self.len0.data_ptr() if self.len0 is not None else None,
+                             self.gen.data_ptr() if self.gen is not None else None,
+                             self.slot_ring.data_ptr() if self.slot_ring is not None else None)
 
 
-def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=None) -> Cache:
+def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=None,
+                evict_distance: int = 0) -> Cache:
     """total_rows: host-known upper bound on the retained rows of all samples."""
     nseg = shape.batch * shape.layers
     dt = torch.float32 if shape.dtype == F32 else torch.bfloat16
@@ -180,7 +190,12 @@ def alloc_cache(shape: Shape, total_rows: int, decode_cap: int, device, fill=Non
     return Cache(mk(cap_rows, shape.heads, shape.head_dim), mk(cap_rows, shape.heads, shape.head_dim),
                  torch.zeros(nseg + 1, dtype=torch.int64, device=device),
                  torch.zeros(nseg, dtype=torch.int32, device=device),
-                 torch.zeros(nseg, dtype=torch.int32, device=device), cap_rows, int(decode_cap))
+                 torch.zeros(nseg, dtype=torch.int32, device=device), cap_rows, int(decode_cap),
+                 int(evict_distance),
+                 torch.zeros(nseg, dtype=torch.int32, device=device) if evict_distance > 0 else None,
+                 torch.zeros(nseg, dtype=torch.int32, device=device) if evict_distance > 0 else None,
+                 torch.full((nseg, evict_distance + 1), -1, dtype=torch.int32, device=device)
+                 if evict_distance > 0 else None)
 
 
 def prefixkv_compact(shape, k, v, order, length, cache: Cache, dev_status, ws, kept=None):

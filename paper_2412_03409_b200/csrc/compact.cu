@@ -13,7 +13,8 @@ __global__ void __launch_bounds__(1024)
 compact_plan_kernel(const int32_t *__restrict__ order, const int32_t *__restrict__ len_in, int nseg,
                     int L, int N, int decode_cap, int64_t total_cap_rows,
                     int64_t *__restrict__ row_offset, int32_t *__restrict__ len_out,
-                    int32_t *__restrict__ cap_out, int32_t *__restrict__ kept, int32_t *dev_status)
+                    int32_t *__restrict__ cap_out, int32_t *__restrict__ kept, int32_t *dev_status,
+                    int32_t *len0, int32_t *gen, int32_t *slot_ring, int ring_size)
 {
     __shared__ uint32_t bitmap[kMaxPromptLen / 32];
     __shared__ int64_t red[32];
@@ -51,7 +52,11 @@ compact_plan_kernel(const int32_t *__restrict__ order, const int32_t *__restrict
         if (seg == nseg - 1) row_offset[nseg] = off + cap;
         len_out[seg] = fits ? n : 0;
         cap_out[seg] = fits ? cap : 0;
+        if (len0) len0[seg] = fits ? n : 0;
+        if (gen) gen[seg] = 0;
     }
+    if (slot_ring)
+        for (int i = tid; i < ring_size; i += blockDim.x) slot_ring[(size_t)seg * ring_size + i] = -1;
     if (!fits) n = 0;
 
     const int32_t *ord = order + (size_t)seg * N;
@@ -160,10 +165,16 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
         if (!ws || !aligned(ws, kWsAlign) || ws_bytes < need) return PKV_ERR_WORKSPACE;
         kept = (int32_t *)ws;
     }
+    if (cache->evict_distance < 0) return PKV_ERR_INVALID_ARG;
+    const bool pruning = cache->evict_distance > 0;
+    if (pruning && (!cache->len0 || !cache->gen || !cache->slot_ring)) return PKV_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     compact_plan_kernel<<<nseg, 1024, 0, stream>>>(order, len, nseg, L, N, cache->decode_cap,
                                                    cache->total_cap_rows, cache->row_offset,
-                                                   cache->len, cache->cap, kept, dev_status);
+                                                   cache->len, cache->cap, kept, dev_status, pruning ? cache->len0 : nullptr,
+                                                   pruning ? cache->gen : nullptr,
+                                                   pruning ? cache->slot_ring : nullptr,
+                                                   cache->evict_distance + 1);
     int rc = check_launch("compact_plan_kernel");
     if (rc != PKV_OK) return rc;
 

@@ -210,6 +210,9 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
         return PKV_ERR_INVALID_ARG;
     if (layer_begin < 0 || layer_end > shape->layers || layer_begin >= layer_end)
         return PKV_ERR_INVALID_ARG;
+    if (cache->evict_distance < 0 ||
+        (cache->evict_distance > 0 && (!cache->len0 || !cache->gen || !cache->slot_ring)))
+        return PKV_ERR_INVALID_ARG;
     if (!shape_supported(shape)) return PKV_ERR_UNSUPPORTED;
     if (!aligned(q, 16) || !aligned(k_new, 16) || !aligned(v_new, 16) || !aligned(out, 16) ||
         !aligned(cache->k, 16) || !aligned(cache->v, 16))
@@ -222,6 +225,7 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
                                       layer_end, out, dev_status, ws, st);
         if (rc >= 0) return rc;  // -1: shape outside the streaming kernel, use the two-kernel path
     }
+    if (cache->evict_distance != 0) return PKV_ERR_UNSUPPORTED;  // pruning lives in the streaming kernel
 #define PKV_DEC(T, D)                                                                              \
     return launch_decode<T, D>(shape, cache, q, k_new, v_new, layer_scale, layer_begin, layer_end, \
                                out, dev_status, ws, st)

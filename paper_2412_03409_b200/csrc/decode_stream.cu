@@ -37,6 +37,10 @@ struct DecodeArgs {
     float *scratch;   // partial slots
     int *plan;        // [nact] int4 records written by the stream kernel for the merge kernel
     int32_t *dev_status;
+    const int32_t *len0;  // [B*L] rows kept by compaction        } only with
+    int32_t *gen;         // [B*L] tokens decoded so far          } decode-time
+    int32_t *slot_ring;   // [B*L][distance + 1] rows of recent tokens } pruning
+    int evict_distance, N;
     int L, H, layer_begin, nl, nact, nseg_total, nstages, nwarps;
     uint32_t row_bytes;
     int64_t total_cap_rows;
@@ -143,15 +147,43 @@ __device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, bool 
     }
 }
 
-// Rows of active segment si that this step attends over besides the appended one, or -1
-// when the segment cannot take another row (full, never compacted, or outside the cache).
-__device__ __forceinline__ int segment_rows(const DecodeArgs &a, int si, int64_t *off_out = nullptr)
+// What this step does to active segment si: the rows it attends over (the new row included),
+// or -1 when the segment cannot take the row (full, never compacted, or outside the cache);
+// the row the new token is written to; the length afterwards.  Without decode-time pruning
+// the new row is appended.  With it (Sec. 3.1: prune at a fixed distance to the latest token,
+// keep the layer's proportion): when generated token g would push the layer past
+// floor(len0 * (N + g + 1) / N) rows and token g - distance is still cached, the new row
+// takes that token's slot instead and the length stays.
+struct SegPlan {
+    int rows, dst, len_after;
+    bool evict;
+    int64_t off;
+};
+__device__ __forceinline__ SegPlan segment_plan(const DecodeArgs &a, int si)
 {
     const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
     const int ln = a.len[seg], cp = a.cap[seg];
-    const int64_t off = a.row_offset[seg];
-    if (off_out) *off_out = off;
-    return (ln >= 1 && ln < cp && off >= 0 && off + cp <= a.total_cap_rows) ? ln : -1;
+    SegPlan p;
+    p.off = a.row_offset[seg];
+    p.evict = false;
+    p.dst = ln;
+    bool ok = ln >= 1 && p.off >= 0 && p.off + cp <= a.total_cap_rows && ln <= cp;
+    const int d = a.evict_distance;
+    if (ok && d > 0) {
+        const int g = a.gen[seg];
+        const int64_t target = ((int64_t)a.len0[seg] * ((int64_t)a.N + g + 1)) / a.N;
+        if ((int64_t)ln + 1 > target && g >= d) {
+            const int r = a.slot_ring[(size_t)seg * (d + 1) + (g - d) % (d + 1)];
+            if (r >= 0 && r < ln) {
+                p.evict = true;
+                p.dst = r;
+            }
+        }
+    }
+    if (!p.evict && ln >= cp) ok = false;  // appending needs head-room
+    p.rows = ok ? (p.evict ? ln : ln + 1) : -1;
+    p.len_after = p.rows;
+    return p;
 }
 
 struct Ring {
@@ -190,7 +222,8 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
     uint64_t *qempty = qfull + 2;          // [2]
     int64_t *seg_off = reinterpret_cast<int64_t *>(qempty + 2);  // [nact] first row of the segment
     int *P = reinterpret_cast<int *>(seg_off + a.nact);          // [nact + 1] unit prefix
-    int *seg_n = P + a.nact + 1;                                 // [nact] rows, or -1 when not active
+    int *seg_rows = P + a.nact + 1;                              // [nact] rows attended (new one included), or -1
+    int *seg_dst = seg_rows + a.nact;                            // [nact] row the new token is written to
     __shared__ int s_abort;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -215,11 +248,11 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
     // above overlapped that kernel's tail; its writes (lengths, cache rows) are visible from here.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int si = tid; si < a.nact; si += blockDim.x) {
-        int64_t off;
-        const int rows = segment_rows(a, si, &off);
-        seg_n[si] = rows;
-        seg_off[si] = off;
-        P[si + 1] = rows >= 0 ? (rows + UR) / UR : 0;  // ceil((rows + 1) / UR): the appended row is the last row
+        const SegPlan sp = segment_plan(a, si);
+        seg_rows[si] = sp.rows;
+        seg_dst[si] = sp.dst | (sp.evict ? (1 << 30) : 0);
+        seg_off[si] = sp.off;
+        P[si + 1] = sp.rows > 0 ? (sp.rows + UR - 1) / UR : 0;
     }
     __syncthreads();
     if (warp == 0) {
@@ -243,7 +276,7 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 
     // segments that cannot take another row: report, write zeros
     for (int si = cta; si < a.nact; si += gridDim.x) {
-        if (seg_n[si] >= 0) continue;
+        if (seg_rows[si] >= 0) continue;
         const int b = si / a.nl, seg = b * a.L + a.layer_begin + si % a.nl;
         if (tid == 0) raise_status(a.dev_status, b, PKV_DEV_CAPACITY);
         T *o = reinterpret_cast<T *>(a.out) + (size_t)seg * H * D;
@@ -258,13 +291,13 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         // The plan, for the merge kernel: rows, first contributing CTA and number of contributing
         // CTAs of every active segment.  (That kernel must not rebuild it from len, which it bumps.)
         for (int i = tid; i < a.nact; i += blockDim.x) {
-            const int rows = seg_n[i];
+            const int rows = seg_rows[i];  // = the segment's length after this step
             int first = 0, cnt = 0;
             if (rows >= 0) {
                 first = unit_owner(P[i], upc, rem);
                 cnt = unit_owner(P[i + 1] - 1, upc, rem) - first + 1;
             }
-            reinterpret_cast<int4 *>(a.plan)[i] = make_int4(rows, first, cnt, 0);
+            reinterpret_cast<int4 *>(a.plan)[i] = make_int4(rows, first, cnt, seg_dst[i]);
         }
     }
     if (cta < G) {
@@ -286,7 +319,7 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
             uint32_t qph = 0;
             int si = si0, issued = 0;
             bool dead = false, piece_start = true;
-            int n = 0, r0 = 0, seg = 0;
+            int n = 0, r0 = 0, seg = 0, newrow = 0;
             int64_t off = 0;
             for (int u = u0; u < u1 && !dead; ++u) {
                 if (u >= P[si + 1]) {
@@ -296,7 +329,8 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                 if (piece_start) {
                     piece_start = false;
                     seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-                    n = seg_n[si];
+                    n = seg_rows[si];
+                    newrow = seg_dst[si] & 0x3fffffff;
                     off = seg_off[si];
                     r0 = (u - P[si]) * UR;
                     wait_phase(qempty + qi, qph ^ 1u, dead, &s_abort);
@@ -307,22 +341,28 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                     qi ^= 1;
                     if (qi == 0) qph ^= 1u;
                 }
-                const int from_cache = min(UR, max(n - r0, 0));
-                const bool has_new = r0 + UR > n;  // this unit ends the segment
-                const uint32_t bytes = (uint32_t)(from_cache + (has_new ? 1 : 0)) * rb;
+                const int cnt = min(UR, n - r0);          // rows of this unit
+                const int nd = newrow - r0;               // the new row's place in it, if 0 <= nd < cnt
+                const bool has_new = nd >= 0 && nd < cnt;
+                const int before = has_new ? nd : cnt;    // cached rows in front of it
+                const int after = has_new ? cnt - nd - 1 : 0;  // and behind it (only when a slot is reused)
+                const uint32_t bytes = (uint32_t)cnt * rb;
 #pragma unroll
                 for (int kv = 0; kv < 2; ++kv) {
                     wait_phase(empty + r.slot, r.phase ^ 1u, dead, &s_abort);
                     if (dead) break;
                     unsigned char *dst = ring + (size_t)r.slot * slot_bytes;
                     mbar_expect_tx(full + r.slot, bytes);
-                    if (from_cache > 0)
-                        bulk_load(dst, reinterpret_cast<const unsigned char *>(kv ? a.cv : a.ck) + (size_t)(off + r0) * rb,
-                                  (uint32_t)from_cache * rb, full + r.slot);
+                    const unsigned char *cache = reinterpret_cast<const unsigned char *>(kv ? a.cv : a.ck);
+                    if (before > 0)
+                        bulk_load(dst, cache + (size_t)(off + r0) * rb, (uint32_t)before * rb, full + r.slot);
                     if (has_new)
-                        bulk_load(dst + (size_t)from_cache * rb,
+                        bulk_load(dst + (size_t)nd * rb,
                                   reinterpret_cast<const unsigned char *>(kv ? a.v_new : a.k_new) + (size_t)seg * rb, rb,
                                   full + r.slot);
+                    if (after > 0)
+                        bulk_load(dst + (size_t)(nd + 1) * rb, cache + (size_t)(off + r0 + nd + 1) * rb,
+                                  (uint32_t)after * rb, full + r.slot);
                     r.advance();
                     ++issued;
                 }
@@ -344,7 +384,7 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         uint32_t qph = 0;
         int si = si0;
         bool dead = false, piece_start = true;
-        int n = 0, r0 = 0, seg = 0, seg_last_u = 0;
+        int n = 0, r0 = 0, seg = 0, seg_last_u = 0, newrow = 0;
         int64_t off = 0;
         size_t seg_vec = 0;
         for (int u = u0; u < u1; ++u) {
@@ -355,7 +395,8 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                 piece_start = false;
                 while (u >= P[si + 1]) ++si;
                 seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
-                n = seg_n[si];
+                n = seg_rows[si];
+                newrow = seg_dst[si] & 0x3fffffff;
                 off = seg_off[si];
                 r0 = (u - P[si]) * UR;
                 seg_last_u = P[si + 1] - 1;
@@ -384,9 +425,10 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                 qi ^= 1;
                 if (qi == 0) qph ^= 1u;
             }
-            const int cnt = min(UR, n + 1 - r0);  // rows of this unit, the appended row included
-            const int new_idx = n - r0;           // its index in the unit when 0 <= new_idx < UR
-            const bool seg_end = new_idx < UR;
+            const int cnt = min(UR, n - r0);      // rows of this unit, the new row included
+            const int new_idx = newrow - r0;      // the new row's index in the unit when 0 <= new_idx < cnt
+            const bool has_new = new_idx >= 0 && new_idx < cnt;
+            const bool seg_end = u == seg_last_u;
             float s[HPW][RPG];
             const bool whole = cnt == UR;  // every row of the unit is valid (uniform over the CTA)
 
@@ -422,9 +464,9 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                     for (int j = 0; j < RPG; ++j)
 #pragma unroll
                         for (int hh = 0; hh < HPW; ++hh) s[hh][j] += __shfl_xor_sync(0xffffffffu, s[hh][j], o);
-                if (seg_end) {  // append: this warp's heads of the new K row go to cache row n
+                if (has_new) {  // this warp's heads of the new K row go to their cache row
                     const unsigned char *src = kb + (uint32_t)new_idx * rb + (uint32_t)h0 * D * sizeof(T);
-                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.ck) + (size_t)(off + n) * rb +
+                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.ck) + (size_t)(off + newrow) * rb +
                                          (size_t)h0 * D * sizeof(T);
                     for (int x = lane; x < HPW * (int)(D * sizeof(T) / 16); x += 32)
                         *reinterpret_cast<uint4 *>(dst + x * 16) = *reinterpret_cast<const uint4 *>(src + x * 16);
@@ -477,9 +519,9 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                         }
                     }
                 }
-                if (seg_end) {
+                if (has_new) {
                     const unsigned char *src = vb + (uint32_t)new_idx * rb + (uint32_t)h0 * D * sizeof(T);
-                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.cv) + (size_t)(off + n) * rb +
+                    unsigned char *dst = reinterpret_cast<unsigned char *>(a.cv) + (size_t)(off + newrow) * rb +
                                          (size_t)h0 * D * sizeof(T);
                     for (int x = lane; x < HPW * (int)(D * sizeof(T) / 16); x += 32)
                         *reinterpret_cast<uint4 *>(dst + x * 16) = *reinterpret_cast<const uint4 *>(src + x * 16);
@@ -566,7 +608,17 @@ __global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
     const int4 rec = reinterpret_cast<const int4 *>(a.plan)[si];
     const int n = rec.x, c_first = rec.y, ncontrib = rec.z;
     if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
-    if (h == 0 && lane == 0) a.len[seg] = n + 1;
+    if (h == 0 && lane == 0) {
+        a.len[seg] = n;  // the record holds the length after this step
+        const int d = a.evict_distance;
+        if (d > 0) {     // only this thread touches the segment's token count and slot ring
+            const int g = a.gen[seg], dst = rec.w & 0x3fffffff;
+            int32_t *ring = a.slot_ring + (size_t)seg * (d + 1);
+            if (rec.w >> 30) ring[(g - d) % (d + 1)] = -1;  // the token d steps back gave up its slot
+            ring[g % (d + 1)] = dst;
+            a.gen[seg] = g + 1;
+        }
+    }
     if (ncontrib == 1) return;
     const size_t cstride = (size_t)a.H * kSlotStride;
     const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;
@@ -621,7 +673,7 @@ size_t decode_stream_ws_bytes(const pkv_shape *s)
 static size_t stream_smem_bytes(int nstages, int ur, uint32_t rb, int nact)
 {
     return (size_t)nstages * ur * rb + 2 * (size_t)rb + (2 * kMaxStages + 4) * sizeof(uint64_t) +
-           (size_t)nact * sizeof(int64_t) + (size_t)(2 * nact + 1) * sizeof(int) + 32;
+           (size_t)nact * sizeof(int64_t) + (size_t)(3 * nact + 1) * sizeof(int) + 32;
 }
 
 template <typename T, int D, int LPR, int HPW, int UR, int MAXT>
@@ -705,6 +757,9 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     a.L = s->layers; a.H = H; a.layer_begin = lb; a.nl = nl; a.nact = nact;
     a.nseg_total = s->batch * s->layers; a.nstages = nstages; a.row_bytes = row_bytes;
     a.total_cap_rows = c->total_cap_rows;
+    a.evict_distance = c->evict_distance;
+    a.len0 = c->len0; a.gen = c->gen; a.slot_ring = c->slot_ring;
+    a.N = s->prompt_len;
 
     const bool bf = s->dtype == PKV_BF16;
     const int vec_per_head = D / (int)(16 / es);

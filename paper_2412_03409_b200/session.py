@@ -13,7 +13,7 @@ from . import api
 
 class Session:
     def __init__(self, B, L, H, D, N, dtype, layer_scale, decode_cap, max_budget_rows=None,
-                 device="cuda", poison=False):
+                 device="cuda", poison=False, evict_distance=0):
         self.device = torch.device(device)
         self.shape = api.make_shape(B, L, H, D, N, dtype)
         self.B, self.L, self.H, self.D, self.N, self.dtype = B, L, H, D, N, dtype
@@ -33,7 +33,8 @@ class Session:
         self.ws_decode = api.alloc_workspace(self.shape, api.WS_DECODE, dev)
         rows = L * N if max_budget_rows is None else min(int(max_budget_rows), L * N)
         self.cache = api.alloc_cache(self.shape, B * rows, decode_cap, dev,
-                                     fill=float("nan") if poison else None)
+                                     fill=float("nan") if poison else None,
+                                     evict_distance=evict_distance)
         self.out = torch.empty((B, L, H, D), dtype=dtype, device=dev)
 
     # -- compress ---------------------------------------------------------

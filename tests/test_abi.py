@@ -64,7 +64,7 @@ def test_null_and_range_arguments_rejected_on_host(api):
         api.PKV_ERR_INVALID_ARG
     assert lib.prefixkv_compact(sh, None, z, None, z, None, None, None, None, None, None, 0, None) == \
         api.PKV_ERR_INVALID_ARG
-    cache = api.CacheStruct(16, 16, 16, 16, 16, 10, 1)
+    cache = api.CacheStruct(16, 16, 16, 16, 16, 10, 1, 0, None, None, None)
     assert lib.prefixkv_decode_attn(sh, ctypes.byref(cache), 16, 16, 16, 16, 1, 1, 16, 16, None, 0,
                                     None) == api.PKV_ERR_INVALID_ARG   # empty layer range
     assert lib.prefixkv_decode_attn(sh, ctypes.byref(cache), 16, 16, 16, 16, 0, 2, 16, 16, None, 0,

@@ -410,3 +410,55 @@ def test_rescale_and_offline_configuration(api):
     # too small a budget is reported
     api.prefixkv_estimate_config(s.shape, s.len, L - 1, cfg, s.status)
     assert s.status[0].item() == api.DEV_BUDGET_TOO_SMALL
+
+
+# --------------------------------------------------------------------------
+# decode-time pruning at a fixed distance (keeps each layer's proportion)
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("name,kw,d", [
+    ("llava7b_b1", dict(B=2, L=3, H=4, N=96, T=40), 4),
+    ("tiny", dict(T=30), 2),
+    ("llava7b_b1", dict(L=2, H=8, N=200, T=24), 9),
+])
+def test_decode_time_pruning_matches_oracle(api, name, kw, d):
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 40) for b in range(w.B)])
+    budgets = [w.budget_rows()] * w.B
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T, evict_distance=d)
+    s.search(torch.tensor(budgets), scores=torch.from_numpy(scores).cuda())
+    s.compact(k, v)
+    ref_sel = oracle_select(scores, budgets)
+    state = {}
+    for b in range(w.B):
+        order, _, res = ref_sel[b]
+        for l in range(w.L):
+            kept = oracle.retained_positions(order[l], res.len[l])
+            state[(b, l)] = dict(k=list(oracle.gather_rows(to_np32(k[b, l]), kept)),
+                                 v=list(oracle.gather_rows(to_np32(v[b, l]), kept)),
+                                 len0=int(res.len[l]), ring=np.full(d + 1, -1, np.int32))
+    dropped = 0
+    for g in range(w.T):
+        qd, kn, vn = wl.make_decode_inputs(w, g, "cuda")
+        got = to_np32(s.decode(qd, kn, vn))
+        lens = s.cache.len.cpu().numpy()
+        for (b, l), st in state.items():
+            dst, ev, n_after = oracle.decode_slot(st["len0"], w.N, g, len(st["k"]), d, st["ring"])
+            if ev:
+                st["k"][dst], st["v"][dst] = to_np32(kn[b, l]), to_np32(vn[b, l])
+                dropped += 1
+            else:
+                st["k"].append(to_np32(kn[b, l])); st["v"].append(to_np32(vn[b, l]))
+            assert lens[b * w.L + l] == n_after == len(st["k"])
+            ref = oracle.decode_attn(to_np32(qd[b, l]), np.stack(st["k"]), np.stack(st["v"]), float(scale[l]))
+            assert np.isfinite(got[b, l]).all()
+            assert np.abs(got[b, l] - ref).max() <= DECODE_TOL[w.dtype]
+    assert dropped > 0 and s.status.cpu().tolist() == [0] * w.B
+    # the cache holds exactly the oracle's rows, slot for slot
+    offs = s.cache.row_offset.cpu().numpy()
+    for (b, l), st in state.items():
+        o = int(offs[b * w.L + l])
+        np.testing.assert_array_equal(to_np32(s.cache.k[o:o + len(st["k"])]), np.stack(st["k"]))
+        np.testing.assert_array_equal(to_np32(s.cache.v[o:o + len(st["v"])]), np.stack(st["v"]))
+        assert int(s.cache.gen[b * w.L + l]) == w.T

@@ -64,7 +64,7 @@ def test_static_scratch_decode_refuses_large_shapes():
     from paper_2412_03409_b200 import api
     big = api.make_shape(16, 32, 32, 128, 640, torch.bfloat16)
     assert api.prefixkv_workspace_bytes(big, api.WS_DECODE) > api.prefixkv_decode_static_limit_bytes()
-    cache = api.CacheStruct(16, 16, 16, 16, 16, 10, 1)
+    cache = api.CacheStruct(16, 16, 16, 16, 16, 10, 1, 0, None, None, None)
     rc = api.lib().prefixkv_decode_attn_static(big, cache, 16, 16, 16, 16, 0, 32, 16, 16, None)
     assert rc == api.PKV_ERR_STATIC_LIMIT
     assert b"16 MiB" in api.lib().prefixkv_last_cuda_error()
