@@ -63,6 +63,9 @@ WORKLOADS = {
                            seed=4, key_bias=True),
 }
 ORDER = ["tiny", "llava7b_b1", "llava7b_b16", "llava13b_b8", "longctx_b4"]
+# A 4-sample cut of llava7b_b16, small enough (2 GB) for multi-pass profiler captures.
+WORKLOADS["llava7b_b4"] = Workload("llava7b_b4", 4, 32, 32, 128, 640, torch.bfloat16, (0.2,), 64, seed=2,
+                                   text_head=32, text_tail=32)
 
 
 def scaled(w: Workload, **kw) -> Workload:
