@@ -14,9 +14,10 @@
 // writes its output directly; one that covers part of it leaves an
 // un-normalised partial in scratch.  A small second kernel, launched as a
 // programmatic dependent so that its launch overlaps the stream, merges the
-// partials of split segments in parallel over all SMs and bumps the lengths.
-#include <cstdlib>
-
+// partials of split segments in parallel over all SMs and writes the lengths.
+// (Merging inside the stream kernel instead, by the last CTA to arrive at a
+// counter, was measured slower: its fence, counter and loads wait behind the
+// other CTAs' bulk traffic, while the second kernel finds the memory system idle.)
 #include "common.cuh"
 
 namespace pkv {
@@ -590,74 +591,138 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 
 }
 
-// Merge kernel: one warp per (head, active segment), launched as a programmatic dependent of
-// the stream kernel, whose CTA 0 leaves it one record per segment (rows, first contributing CTA,
-// number of contributors).  For a segment split over several CTAs it combines their partials,
-// up to 16 contributors per round trip; for every segment that took a row, the warp of head 0
-// bumps len.  It reads len nowhere: blocks of a large grid start after others have bumped it.
-template <typename T, int D>
-__global__ void __launch_bounds__(32) decode_finish_kernel(const DecodeArgs a)
-{
-    constexpr int kSlotStride = D + 4;
-    constexpr int KB = 16;  // contributors per batch
-    const int h = blockIdx.x, si = blockIdx.y, lane = threadIdx.x;
+template <typename T, int E> struct Pack;
+template <> struct Pack<float, 4> {
+    __device__ static void store(float *dst, const float *x) { *reinterpret_cast<float4 *>(dst) = make_float4(x[0], x[1], x[2], x[3]); }
+};
+template <> struct Pack<float, 2> {
+    __device__ static void store(float *dst, const float *x) { *reinterpret_cast<float2 *>(dst) = make_float2(x[0], x[1]); }
+};
+template <> struct Pack<__nv_bfloat16, 4> {
+    __device__ static void store(__nv_bfloat16 *dst, const float *x)
+    {
+        __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+        *reinterpret_cast<uint2 *>(dst) =
+            make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+    }
+};
+template <> struct Pack<__nv_bfloat16, 2> {
+    __device__ static void store(__nv_bfloat16 *dst, const float *x)
+    {
+        *reinterpret_cast<__nv_bfloat162 *>(dst) = __floats2bfloat162_rn(x[0], x[1]);
+    }
+};
+template <int E> struct LoadF;
+template <> struct LoadF<4> {
+    __device__ static void ld(const float *p, float *x)
+    {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(p));
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+};
+template <> struct LoadF<2> {
+    __device__ static void ld(const float *p, float *x)
+    {
+        const float2 v = __ldcg(reinterpret_cast<const float2 *>(p));
+        x[0] = v.x; x[1] = v.y;
+    }
+};
 
-    const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+// Merge kernel, launched as a programmatic dependent of the stream kernel, whose CTA 0 leaves
+// it one record per active segment (length after the step, first contributing CTA, number of
+// contributors, row written).  Every block copies the records to shared memory; its warps then
+// take (segment, group of HG heads) items in a grid-stride loop and, for a segment split over
+// several CTAs, combine the partials -- lane x holds elements [x * D / 32, (x + 1) * D / 32) of
+// a head, and HG heads x KB contributors are in flight before any is used.  One thread per
+// segment writes the new length.  Nothing here reads len: blocks of one grid start at different
+// times.
+constexpr int kFinishWarps = 8;
+template <typename T, int D, int HG>
+__global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_kernel(const DecodeArgs a)
+{
+    constexpr int kSlotStride = D + 4, EPM = D / 32, KB = 8 / HG;
+    __shared__ int4 rec[kMaxActive];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // e.g. the next decode step
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
-    const int4 rec = reinterpret_cast<const int4 *>(a.plan)[si];
-    const int n = rec.x, c_first = rec.y, ncontrib = rec.z;
-    if (n < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
-    if (h == 0 && lane == 0) {
-        a.len[seg] = n;  // the record holds the length after this step
+    for (int i = tid; i < a.nact; i += blockDim.x) rec[i] = reinterpret_cast<const int4 *>(a.plan)[i];
+    __syncthreads();
+
+    for (int si = blockIdx.x * blockDim.x + tid; si < a.nact; si += gridDim.x * blockDim.x) {
+        const int4 r = rec[si];
+        if (r.x < 0) continue;  // could not take a row: reported and zero-filled by the stream kernel
+        const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+        a.len[seg] = r.x;
         const int d = a.evict_distance;
-        if (d > 0) {     // only this thread touches the segment's token count and slot ring
-            const int g = a.gen[seg], dst = rec.w & 0x3fffffff;
+        if (d > 0) {  // only this thread touches the segment's token count and slot ring
+            const int g = a.gen[seg];
             int32_t *ring = a.slot_ring + (size_t)seg * (d + 1);
-            if (rec.w >> 30) ring[(g - d) % (d + 1)] = -1;  // the token d steps back gave up its slot
-            ring[g % (d + 1)] = dst;
+            if (r.w >> 30) ring[(g - d) % (d + 1)] = -1;  // the token d steps back gave up its slot
+            ring[g % (d + 1)] = r.w & 0x3fffffff;
             a.gen[seg] = g + 1;
         }
     }
-    if (ncontrib == 1) return;
+
+    const int groups = a.H / HG;
     const size_t cstride = (size_t)a.H * kSlotStride;
-    const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;
-    float M = -INFINITY, z = 0.f, o[D / 32];
+    for (int item = blockIdx.x * kFinishWarps + warp; item < a.nact * groups; item += gridDim.x * kFinishWarps) {
+        const int si = item / groups, h0 = (item - si * groups) * HG;
+        const int4 r = rec[si];
+        const int c_first = r.y, ncontrib = r.z;
+        if (r.x < 0 || ncontrib <= 1) continue;
+        const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+        const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h0) * kSlotStride;
+        float M[HG], z[HG], o[HG][EPM];
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) o[i] = 0.f;
-    for (int k0 = 0; k0 < ncontrib; k0 += KB) {
-        float w[KB], ls[KB], x[KB][D / 32];
+        for (int hh = 0; hh < HG; ++hh) {
+            M[hh] = -INFINITY;
+            z[hh] = 0.f;
 #pragma unroll
-        for (int kk = 0; kk < KB; ++kk) {  // every load of the batch is in flight before any use
-            const float *sl = base + min(k0 + kk, ncontrib - 1) * cstride;
-            w[kk] = sl[D];
-            ls[kk] = sl[D + 1];
-#pragma unroll
-            for (int i = 0; i < D / 32; ++i) x[kk][i] = sl[lane + 32 * i];
+            for (int i = 0; i < EPM; ++i) o[hh][i] = 0.f;
         }
-        float mb = M;
+#pragma unroll 1
+        for (int k0 = 0; k0 < ncontrib; k0 += KB) {
+            float2 ml[HG][KB];
+            float x[HG][KB][EPM];
 #pragma unroll
-        for (int kk = 0; kk < KB; ++kk)
-            if (k0 + kk < ncontrib) mb = fmaxf(mb, w[kk]);
-        const float corr = M == -INFINITY ? 0.f : exp2f(M - mb);
-        z *= corr;
+            for (int kk = 0; kk < KB; ++kk) {
+                const float *sl = base + (size_t)min(k0 + kk, ncontrib - 1) * cstride;
 #pragma unroll
-        for (int i = 0; i < D / 32; ++i) o[i] *= corr;
-        M = mb;
+                for (int hh = 0; hh < HG; ++hh) {
+                    ml[hh][kk] = *reinterpret_cast<const float2 *>(sl + hh * kSlotStride + D);
+                    LoadF<EPM>::ld(sl + hh * kSlotStride + lane * EPM, x[hh][kk]);
+                }
+            }
 #pragma unroll
-        for (int kk = 0; kk < KB; ++kk) {
-            if (k0 + kk < ncontrib) {
-                const float ww = exp2f(w[kk] - M);
-                z = fmaf(ww, ls[kk], z);
+            for (int hh = 0; hh < HG; ++hh) {
+                float mb = M[hh];
 #pragma unroll
-                for (int i = 0; i < D / 32; ++i) o[i] = fmaf(ww, x[kk][i], o[i]);
+                for (int kk = 0; kk < KB; ++kk)
+                    if (k0 + kk < ncontrib) mb = fmaxf(mb, ml[hh][kk].x);
+                const float corr = M[hh] == -INFINITY ? 0.f : exp2f(M[hh] - mb);
+                z[hh] *= corr;
+#pragma unroll
+                for (int i = 0; i < EPM; ++i) o[hh][i] *= corr;
+                M[hh] = mb;
+#pragma unroll
+                for (int kk = 0; kk < KB; ++kk) {
+                    if (k0 + kk < ncontrib) {
+                        const float ww = exp2f(ml[hh][kk].x - mb);
+                        z[hh] = fmaf(ww, ml[hh][kk].y, z[hh]);
+#pragma unroll
+                        for (int i = 0; i < EPM; ++i) o[hh][i] = fmaf(ww, x[hh][kk][i], o[hh][i]);
+                    }
+                }
             }
         }
-    }
-    const float inv = 1.f / z;
-    T *dst = reinterpret_cast<T *>(a.out) + ((size_t)seg * a.H + h) * D;
 #pragma unroll
-    for (int i = 0; i < D / 32; ++i) dst[lane + 32 * i] = from_float<T>(o[i] * inv);
+        for (int hh = 0; hh < HG; ++hh) {
+            const float inv = 1.f / z[hh];
+#pragma unroll
+            for (int i = 0; i < EPM; ++i) o[hh][i] *= inv;
+            Pack<T, EPM>::store(reinterpret_cast<T *>(a.out) + ((size_t)seg * a.H + h0 + hh) * D + lane * EPM, o[hh]);
+        }
+    }
 }
 
 static size_t plan_bytes(int nact) { return round_up((size_t)nact * sizeof(int4), kWsAlign); }
@@ -700,13 +765,18 @@ static int launch_variant(const DecodeArgs &a, int sms, cudaStream_t st)
         set_cuda_error(e, "decode_stream_kernel");
         return PKV_ERR_CUDA;
     }
-    cfg.gridDim = dim3(a.H, a.nact);
-    cfg.blockDim = dim3(32);
+    // One head per warp item while that still fills the GPU once (every partial of a segment is
+    // then in flight at the same time); two heads per item beyond that.
+    const int hg = (a.H % 2 == 0 && a.nact * a.H > 2 * sms * kFinishWarps) ? 2 : 1;
+    const int items = a.nact * (a.H / hg);
+    const int blocks = (items + kFinishWarps - 1) / kFinishWarps;
+    cfg.gridDim = dim3(blocks < sms ? blocks : sms);
+    cfg.blockDim = dim3(kFinishWarps * 32);
     cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D>, a);
+    if (hg == 2)
+        e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D, 2>, a);
+    else
+        e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D, 1>, a);
     if (e != cudaSuccess) {
         set_cuda_error(e, "decode_finish_kernel");
         return PKV_ERR_CUDA;
@@ -767,10 +837,6 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     // state that each SM sub-partition's register file holds its warps.
     int lpr = 8, hpw = H <= 16 ? 1 : (H <= 32 ? 2 : 4);
     if (H > 16 && vec_per_head >= 16) lpr = 16;
-    if (const char *env = getenv("PKV_DECODE_VARIANT")) {
-        int code = atoi(env);
-        if (code > 0) { lpr = code / 10; hpw = code % 10; }
-    }
     if (vec_per_head < lpr || H % hpw != 0) return -1;
     a.nwarps = H / hpw;
 #define PKV_V(T, DD, LPR, HPW, UR, MAXT)                                       \
