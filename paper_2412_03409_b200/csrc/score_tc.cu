@@ -135,6 +135,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64])
+{
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
 // 2^x on the special-function unit, one instruction (inputs here are <= 0 or -inf; flushing
 // denormal results to zero is harmless for sums of probabilities).
 __device__ __forceinline__ float ex2(float x)
@@ -158,11 +169,62 @@ struct Ring2 {
     }
 };
 
+// Pass 1 on NC consecutive logits of one query row: running maximum and sum in the log2
+// domain.  Four interleaved chains each for the maximum and the sum: with two reader warps per
+// scheduler a long dependent chain would leave it idle.  `fast` (scale > 0, the usual case):
+// the extreme of sc * x is sc * max x, so masked logits may stay -inf.
+template <int NC>
+__device__ __forceinline__ void lse_block(float (&v)[NC], float sc, bool fast, float &run_max, float &run_sum)
+{
+    if (!fast) {
+#pragma unroll
+        for (int i = 0; i < NC; ++i) v[i] = v[i] == -INFINITY ? -INFINITY : v[i] * sc;
+    }
+    float c4[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+    for (int i = 4; i < NC; ++i) c4[i & 3] = fmaxf(c4[i & 3], v[i]);
+    const float cmax = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
+    const float nm = fmaxf(run_max, fast ? cmax * sc : cmax);  // finite: column 0 is never masked
+    float p4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (fast) {
+#pragma unroll
+        for (int i = 0; i < NC; ++i) p4[i & 3] += ex2(fmaf(v[i], sc, -nm));
+    } else {
+#pragma unroll
+        for (int i = 0; i < NC; ++i) p4[i & 3] += ex2(v[i] - nm);
+    }
+    run_sum = fmaf(run_sum, ex2(run_max - nm), (p4[0] + p4[1]) + (p4[2] + p4[3]));
+    run_max = nm;
+}
+
+// Pass 2 on the logits of NC consecutive queries against one key: sum of the probabilities,
+// lse = the queries' normalisers (shared memory, log2 domain).  On the block the causal boundary
+// crosses (`edge`) query i of the block counts only when i >= lane.
+template <int NC>
+__device__ __forceinline__ float colsum_block(const float (&v)[NC], const float *lse, float sc, bool edge, int lane)
+{
+    const float4 *lp = reinterpret_cast<const float4 *>(lse);
+    float p4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i4 = 0; i4 < NC / 4; ++i4) {
+        const float4 ls = lp[i4];
+        const float lv[4] = {ls.x, ls.y, ls.z, ls.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i4 * 4 + u;
+            const float p = ex2(fmaf(v[i], sc, -lv[u]));
+            p4[u] += (!edge || i >= lane) ? p : 0.f;
+        }
+    }
+    return (p4[0] + p4[1]) + (p4[2] + p4[3]);
+}
+
 // Work item w -> (segment-head sh, tile t).  The tiles of one head are consecutive items, so
 // the CTAs running at any moment share a few dozen heads whose Q and K stay in L2 and every
 // operand byte comes from HBM once per pass.  Pass 2 walks the heads backwards: it starts on
-// what pass 1 touched last.  A CTA's successive items (stride gridDim.x) cycle through the
-// tile index, which mixes long and short items evenly.
+// what pass 1 touched last.  A CTA's successive items (stride gridDim.x, chosen by the launcher to
+// share no factor with the tiles per head) cycle through the tile index, which mixes long and
+// short items evenly.
 template <int PASS> __device__ __forceinline__ void decode_item(int w, int nsh, int tiles, int &sh, int &t)
 {
     const int q = w / tiles;
@@ -314,55 +376,33 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // blocks 0..quarter in pass 1 (keys <= query), quarter..3 in pass 2 (queries >= key).
                 const int c_lo = (PASS == 2 && diag) ? quarter : 0;
                 const int c_hi = (PASS == 1 && diag) ? quarter : TT / 32 - 1;
+                if (!diag) {
+                    // a full tile: two 64-column loads, so that the accumulator's read latency is paid
+                    // twice per tile
 #pragma unroll 1
-                for (int cblk = c_lo; cblk <= c_hi; ++cblk) {
-                    float v[32];
-                    tmem_ld32(taddr + cblk * 32, v);
-                    const bool edge = diag && cblk == quarter;  // the block the causal boundary crosses
-                    if (PASS == 1) {
-                        if (edge) {
+                    for (int half = 0; half < 2; ++half) {
+                        float v[64];
+                        tmem_ld64(taddr + half * 64, v);
+                        if (PASS == 1)
+                            lse_block<64>(v, sc, fast, run_max, run_sum);
+                        else
+                            col_sum += colsum_block<64>(v, &s_lse[rs.idx][half * 64], sc, false, lane);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int cblk = c_lo; cblk <= c_hi; ++cblk) {
+                        float v[32];
+                        tmem_ld32(taddr + cblk * 32, v);
+                        const bool edge = cblk == quarter;  // the block the causal boundary crosses
+                        if (PASS == 1) {
+                            if (edge) {
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = i <= lane ? v[i] : -INFINITY;
-                        }
-                        if (fast) {
-                            float cmax = v[0];
-#pragma unroll
-                            for (int i = 1; i < 32; ++i) cmax = fmaxf(cmax, v[i]);
-                            const float nm = fmaxf(run_max, cmax * sc);  // finite: column 0 is never masked
-                            float part = 0.f;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) part += ex2(fmaf(v[i], sc, -nm));
-                            run_sum = fmaf(run_sum, ex2(run_max - nm), part);
-                            run_max = nm;
+                                for (int i = 0; i < 32; ++i) v[i] = i <= lane ? v[i] : -INFINITY;
+                            }
+                            lse_block<32>(v, sc, fast, run_max, run_sum);
                         } else {
-                            float cmax = -INFINITY;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                v[i] = v[i] == -INFINITY ? -INFINITY : v[i] * sc;
-                                cmax = fmaxf(cmax, v[i]);
-                            }
-                            const float nm = fmaxf(run_max, cmax);
-                            float part = 0.f;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) part += ex2(v[i] - nm);
-                            run_sum = fmaf(run_sum, ex2(run_max - nm), part);
-                            run_max = nm;
+                            col_sum += colsum_block<32>(v, &s_lse[rs.idx][cblk * 32], sc, edge, lane);
                         }
-                    } else {
-                        const float4 *lp = reinterpret_cast<const float4 *>(&s_lse[rs.idx][cblk * 32]);
-                        float part = 0.f;
-#pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            const float4 ls = lp[i4];
-                            const float lv[4] = {ls.x, ls.y, ls.z, ls.w};
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const int i = i4 * 4 + u;
-                                const float p = ex2(fmaf(v[i], sc, -lv[u]));
-                                part += (!edge || i >= lane) ? p : 0.f;
-                            }
-                        }
-                        col_sum += part;
                     }
                 }
                 fence_before();
@@ -450,7 +490,15 @@ int launch_pass(const CUtensorMap &mq, const CUtensorMap &mk, const ScoreArgs &a
     int rc = ensure_dynamic_smem((const void *)score_tile_kernel<PASS, D>, (int)smem, done);
     if (rc != PKV_OK) return rc;
     const int items = a.nseg * a.H * a.tiles;
-    const int grid = items < 2 * sms ? items : 2 * sms;
+    // A CTA takes items blockIdx.x, + grid, + 2 grid, ...: with a grid size that shares no factor
+    // with the tiles per head its items run through every tile index (long and short items) evenly.
+    // (296 CTAs and 16 tiles share 8: every CTA would see two tile indices only, and the slowest
+    // would do 12 tiles per item against a mean of 8.5.)
+    int grid = items < 2 * sms ? items : 2 * sms;
+    if (items > grid) {
+        auto gcd = [](int x, int y) { while (y) { int r = x % y; x = y; y = r; } return x; };
+        while (grid > sms && gcd(grid, a.tiles) != 1) --grid;
+    }
     score_tile_kernel<PASS, D><<<grid, 192, smem, st>>>(mq, mk, a);
     return check_launch(PASS == 1 ? "score_tile_kernel<1>" : "score_tile_kernel<2>");
 }
