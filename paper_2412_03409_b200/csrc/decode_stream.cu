@@ -630,22 +630,36 @@ template <> struct LoadF<2> {
 
 // Merge kernel, launched as a programmatic dependent of the stream kernel, whose CTA 0 leaves
 // it one record per active segment (length after the step, first contributing CTA, number of
-// contributors, row written).  Every block copies the records to shared memory; its warps then
-// take (segment, group of HG heads) items in a grid-stride loop and, for a segment split over
-// several CTAs, combine the partials -- lane x holds elements [x * D / 32, (x + 1) * D / 32) of
-// a head, and HG heads x KB contributors are in flight before any is used.  One thread per
-// segment writes the new length.  Nothing here reads len: blocks of one grid start at different
-// times.
-constexpr int kFinishWarps = 8;
+// contributors, row written).  Every block copies the records to shared memory and lists the
+// segments that were split over several CTAs; its warps then take (split segment, group of HG
+// heads) items in a grid-stride loop and combine the partials -- lane x holds elements
+// [x * D / 32, (x + 1) * D / 32) of a head, and HG heads x KB contributors are in flight before
+// any is used.  One thread per segment writes the new length.  Nothing here reads len: blocks of
+// one grid start at different times.
+constexpr int kFinishWarps = 16;
 template <typename T, int D, int HG>
 __global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_kernel(const DecodeArgs a)
 {
     constexpr int kSlotStride = D + 4, EPM = D / 32, KB = 8 / HG;
     __shared__ int4 rec[kMaxActive];
+    __shared__ short split_seg[kMaxActive];
+    __shared__ int nsplit;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // e.g. the next decode step
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
     for (int i = tid; i < a.nact; i += blockDim.x) rec[i] = reinterpret_cast<const int4 *>(a.plan)[i];
+    __syncthreads();
+    if (warp == 0) {  // the split segments, in order
+        int n = 0;
+        for (int base = 0; base < a.nact; base += 32) {
+            const int i = base + lane;
+            const bool is_split = i < a.nact && rec[i].x >= 0 && rec[i].z > 1;
+            const unsigned m = __ballot_sync(0xffffffffu, is_split);
+            if (is_split) split_seg[n + __popc(m & ((1u << lane) - 1))] = (short)i;
+            n += __popc(m);
+        }
+        if (lane == 0) nsplit = n;
+    }
     __syncthreads();
 
     for (int si = blockIdx.x * blockDim.x + tid; si < a.nact; si += gridDim.x * blockDim.x) {
@@ -665,11 +679,11 @@ __global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_kernel(const 
 
     const int groups = a.H / HG;
     const size_t cstride = (size_t)a.H * kSlotStride;
-    for (int item = blockIdx.x * kFinishWarps + warp; item < a.nact * groups; item += gridDim.x * kFinishWarps) {
-        const int si = item / groups, h0 = (item - si * groups) * HG;
+    for (int item = blockIdx.x * kFinishWarps + warp; item < nsplit * groups; item += gridDim.x * kFinishWarps) {
+        const int sp = item / groups, h0 = (item - sp * groups) * HG;
+        const int si = split_seg[sp];
         const int4 r = rec[si];
         const int c_first = r.y, ncontrib = r.z;
-        if (r.x < 0 || ncontrib <= 1) continue;
         const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
         const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h0) * kSlotStride;
         float M[HG], z[HG], o[HG][EPM];
@@ -767,7 +781,7 @@ static int launch_variant(const DecodeArgs &a, int sms, cudaStream_t st)
     }
     // One head per warp item while that still fills the GPU once (every partial of a segment is
     // then in flight at the same time); two heads per item beyond that.
-    const int hg = (a.H % 2 == 0 && a.nact * a.H > 2 * sms * kFinishWarps) ? 2 : 1;
+    const int hg = (a.H % 2 == 0 && a.nact * a.H > sms * kFinishWarps) ? 2 : 1;
     const int items = a.nact * (a.H / hg);
     const int blocks = (items + kFinishWarps - 1) / kFinishWarps;
     cfg.gridDim = dim3(blocks < sms ? blocks : sms);
