@@ -36,6 +36,32 @@ inline size_t esize(const pkv_shape *s) { return s->dtype == PKV_F32 ? 4 : 2; }
 inline bool aligned(const void *p, size_t a) { return ((uintptr_t)p % a) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Launch as a programmatic dependent of the kernel before it in the stream: the grid may be set
+// up while that kernel drains; the kernel's own griddepcontrol.wait holds it until the earlier
+// kernel has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t st, Args... args)
+{
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+// In a kernel launched that way: wait for the earlier kernel, then let the next one be set up.
+__device__ __forceinline__ void dependent_entry()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // Raise a sample's status word from PKV_DEV_OK; the first condition wins.
 __device__ __forceinline__ void raise_status(int32_t *dev_status, int b, int code)
 {

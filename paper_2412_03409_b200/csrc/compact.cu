@@ -22,6 +22,7 @@ compact_plan_kernel(const int32_t *__restrict__ order, const int32_t *__restrict
     __shared__ int64_t s_off;
     const int seg = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = seg / L;
+    dependent_entry();
 
     auto clamp_len = [&](int v) { return (v < 1 || v > N) ? 0 : v; };
 
@@ -104,6 +105,7 @@ gather_rows_kernel(const uint4 *__restrict__ k, const uint4 *__restrict__ v, pkv
                    int N, int H, uint4 *__restrict__ ck, uint4 *__restrict__ cv)
 {
     const int seg = blockIdx.x;
+    dependent_entry();  // the plan kernel's lists, lengths and offsets are complete
     const int n = len[seg];
     const int b = seg / L, l = seg % L;
     const int64_t off = row_offset[seg];
@@ -169,14 +171,15 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
     const bool pruning = cache->evict_distance > 0;
     if (pruning && (!cache->len0 || !cache->gen || !cache->slot_ring)) return PKV_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    compact_plan_kernel<<<nseg, 1024, 0, stream>>>(order, len, nseg, L, N, cache->decode_cap,
-                                                   cache->total_cap_rows, cache->row_offset,
-                                                   cache->len, cache->cap, kept, dev_status, pruning ? cache->len0 : nullptr,
-                                                   pruning ? cache->gen : nullptr,
-                                                   pruning ? cache->slot_ring : nullptr,
-                                                   cache->evict_distance + 1);
-    int rc = check_launch("compact_plan_kernel");
-    if (rc != PKV_OK) return rc;
+    cudaError_t e = launch_dependent(compact_plan_kernel, dim3(nseg), dim3(1024), 0, stream, order, len, nseg, L, N,
+                                     cache->decode_cap, cache->total_cap_rows, cache->row_offset, cache->len,
+                                     cache->cap, kept, dev_status, pruning ? cache->len0 : nullptr,
+                                     pruning ? cache->gen : nullptr, pruning ? cache->slot_ring : nullptr,
+                                     cache->evict_distance + 1);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "compact_plan_kernel");
+        return PKV_ERR_CUDA;
+    }
 
     pkv_strides k16 = {ks.b / per16, ks.l / per16, ks.h / per16, ks.n / per16};
     pkv_strides v16 = {vs.b / per16, vs.l / per16, vs.h / per16, vs.n / per16};
@@ -185,10 +188,10 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
     if (slices < 1) slices = 1;
     if (slices > N) slices = N;
     dim3 grid(nseg, slices);
-#define PKV_GATHER(V)                                                                             \
-    gather_rows_kernel<V><<<grid, 256, 0, stream>>>((const uint4 *)k, (const uint4 *)v, k16, v16, \
-                                                    kept, cache->len, cache->row_offset, L, N, H, \
-                                                    (uint4 *)cache->k, (uint4 *)cache->v)
+#define PKV_GATHER(V)                                                                                  \
+    e = launch_dependent(gather_rows_kernel<V>, grid, dim3(256), 0, stream, (const uint4 *)k,          \
+                         (const uint4 *)v, k16, v16, (const int32_t *)kept, (const int32_t *)cache->len, \
+                         (const int64_t *)cache->row_offset, L, N, H, (uint4 *)cache->k, (uint4 *)cache->v)
     switch (vph) {
     case 8: PKV_GATHER(8); break;
     case 16: PKV_GATHER(16); break;
@@ -196,5 +199,9 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
     default: return PKV_ERR_UNSUPPORTED;
     }
 #undef PKV_GATHER
-    return check_launch("gather_rows_kernel");
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "gather_rows_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }

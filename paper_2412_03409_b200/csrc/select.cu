@@ -48,6 +48,7 @@ sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t 
     const int nthr = blockDim.x;
     const float *src = scores + (size_t)seg * N;
     if (tid == 0) s_flags = 0;
+    dependent_entry();  // set up while the kernel before it drained; its results are read from here on
 
     bool bad = false;
     for (int i = tid; i < P; i += nthr) {
@@ -128,10 +129,19 @@ sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t 
 // cumulative values below theta, found by a 32-way search (every lane probes
 // one pivot per round), plus one, clamped to [1, N].
 // ---------------------------------------------------------------------------
+// `pivot` is the lane's probe of the first round, c[(lane + 1) * chunk0 - 1] (or ~0 past the
+// end): it does not depend on theta, so a caller that searches one row many times loads it once.
 __device__ __forceinline__ int warp_length_for_theta(const uint64_t *__restrict__ c, int N,
-                                                     uint64_t theta, int lane)
+                                                     uint64_t theta, int lane, uint64_t pivot)
 {
     int a = 0, bnd = N;  // the count lies in [a, bnd]
+    {
+        const int chunk = (N + 31) >> 5;
+        const int k = __popc(__ballot_sync(0xffffffffu, pivot < theta));
+        a = k * chunk;
+        const int nb = (k + 1) * chunk - 1;
+        bnd = nb < N ? nb : N;
+    }
     while (bnd > a) {
         int chunk = (bnd - a + 31) >> 5;
         int idx = a + (lane + 1) * chunk - 1;
@@ -158,19 +168,52 @@ search_kernel(const uint64_t *__restrict__ cum, const int64_t *__restrict__ budg
     const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
     const uint64_t *cb = cum + (size_t)b * L * N;
+    dependent_entry();  // the sort kernel's sums are complete
     const int64_t budget = budget_rows[b];
+
+    // What every midpoint needs of a layer's row and never changes: its total and this lane's
+    // first-round probe.  Kept in registers for the first kHoist layers of the warp.
+    constexpr int kHoist = 4;
+    const int chunk0 = (N + 31) >> 5;
+    double tot_r[kHoist];
+    uint64_t piv_r[kHoist];
+#pragma unroll
+    for (int k = 0; k < kHoist; ++k) {
+        const int l = warp + k * nwarp;
+        tot_r[k] = 0.0;
+        piv_r[k] = ~0ull;
+        if (l < L) {
+            const uint64_t *c = cb + (size_t)l * N;
+            const int idx = (lane + 1) * chunk0 - 1;
+            tot_r[k] = (double)c[N - 1];
+            if (idx < N) piv_r[k] = c[idx];
+        }
+    }
 
     auto eval = [&](double p, int buf) -> int64_t {
         int *dst = s_len + buf * L;
-        for (int l = warp; l < L; l += nwarp) {
+#pragma unroll
+        for (int k = 0; k < kHoist; ++k) {
+            const int l = warp + k * nwarp;
+            if (l < L) {
+                int n = N;
+                if (p < 1.0) {
+                    const uint64_t theta = __double2ull_ru(__dmul_rn(p, tot_r[k]));
+                    n = warp_length_for_theta(cb + (size_t)l * N, N, theta, lane, piv_r[k]);
+                }
+                if (lane == 0) dst[l] = n;
+            }
+        }
+        for (int l = warp + kHoist * nwarp; l < L; l += nwarp) {
             const uint64_t *c = cb + (size_t)l * N;
             int n;
             if (p >= 1.0) {
                 n = N;
             } else {
+                const int idx = (lane + 1) * chunk0 - 1;
                 double total = (double)c[N - 1];
                 uint64_t theta = __double2ull_ru(__dmul_rn(p, total));
-                n = warp_length_for_theta(c, N, theta, lane);
+                n = warp_length_for_theta(c, N, theta, lane, idx < N ? c[idx] : ~0ull);
             }
             if (lane == 0) dst[l] = n;
         }
@@ -252,9 +295,13 @@ static int launch_sort(const pkv_shape *s, const float *scores, int32_t *order, 
         int rc = ensure_dynamic_smem((const void *)sort_scan_kernel, 128 * 1024, attr_done);
         if (rc != PKV_OK) return rc;
     }
-    sort_scan_kernel<<<s->batch * s->layers, nthr, smem, st>>>(scores, N, P, s->layers, order, cum,
-                                                               dev_status);
-    return check_launch("sort_scan_kernel");
+    cudaError_t e = launch_dependent(sort_scan_kernel, dim3(s->batch * s->layers), dim3(nthr), smem, st, scores, N, P,
+                                     (int)s->layers, order, cum, dev_status);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "sort_scan_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
 
 }  // namespace pkv
@@ -278,9 +325,14 @@ extern "C" int prefixkv_search(const pkv_shape *shape, const float *scores,
     clear_status_kernel<<<(B + 255) / 256, 256, 0, st>>>(dev_status, B);
     int rc = launch_sort(shape, scores, order, cum, dev_status, st);
     if (rc != PKV_OK) return rc;
-    search_kernel<<<B, 1024, 2 * L * sizeof(int), st>>>(cum, budget_rows, L, N, tol, max_iters,
-                                                        slack_rows, len, p_out, iters_out, dev_status);
-    return check_launch("search_kernel");
+    cudaError_t e = launch_dependent(search_kernel, dim3(B), dim3(1024), 2 * L * sizeof(int), st,
+                                     (const uint64_t *)cum, budget_rows, L, N, tol, (int)max_iters, slack_rows, len,
+                                     p_out, iters_out, dev_status);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "search_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
 
 extern "C" int prefixkv_apply_lengths(const pkv_shape *shape, const float *scores,
