@@ -211,6 +211,8 @@ int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, cons
  *   q, k_new, v_new, out   [B,L,H,D] contiguous, dtype of the cache
  * A segment already at capacity raises PKV_DEV_CAPACITY, appends nothing and
  * writes zeros.
+ * k_new and v_new may both be NULL: nothing is appended, len stays, and out attends over the
+ * len rows that are there (a second query against the same cache).
  * With cache->evict_distance = d > 0 the layer proportions are kept while decoding (Sec. 3.1,
  * Fig. 2a; the distance and the exact rule are the cited work's, this is the reading): when
  * generated token g would push a layer past floor(len0 * (N + g + 1) / N) rows and token

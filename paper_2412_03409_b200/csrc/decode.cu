@@ -206,7 +206,7 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
                                     void *cuda_stream)
 {
     if (!shape_ok(shape) || !cache || !cache->k || !cache->v || !cache->row_offset || !cache->len ||
-        !cache->cap || !q || !k_new || !v_new || !layer_scale || !out || !dev_status)
+        !cache->cap || !q || (k_new == nullptr) != (v_new == nullptr) || !layer_scale || !out || !dev_status)
         return PKV_ERR_INVALID_ARG;
     if (layer_begin < 0 || layer_end > shape->layers || layer_begin >= layer_end)
         return PKV_ERR_INVALID_ARG;
@@ -226,6 +226,7 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
         if (rc >= 0) return rc;  // -1: shape outside the streaming kernel, use the two-kernel path
     }
     if (cache->evict_distance != 0) return PKV_ERR_UNSUPPORTED;  // pruning lives in the streaming kernel
+    if (!k_new) return PKV_ERR_UNSUPPORTED;                       // and so does attending without appending
 #define PKV_DEC(T, D)                                                                              \
     return launch_decode<T, D>(shape, cache, q, k_new, v_new, layer_scale, layer_begin, layer_end, \
                                out, dev_status, ws, st)

@@ -169,6 +169,12 @@ __device__ __forceinline__ SegPlan segment_plan(const DecodeArgs &a, int si)
     p.evict = false;
     p.dst = ln;
     bool ok = ln >= 1 && p.off >= 0 && p.off + cp <= a.total_cap_rows && ln <= cp;
+    if (!a.k_new) {  // nothing to append: attend over the rows that are there
+        p.dst = 0x3fffffff;
+        p.rows = ok ? ln : -1;
+        p.len_after = p.rows;
+        return p;
+    }
     const int d = a.evict_distance;
     if (ok && d > 0) {
         const int g = a.gen[seg];
@@ -667,7 +673,7 @@ __global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_kernel(const 
         if (r.x < 0) continue;  // could not take a row: reported and zero-filled by the stream kernel
         const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
         a.len[seg] = r.x;
-        const int d = a.evict_distance;
+        const int d = a.k_new ? a.evict_distance : 0;
         if (d > 0) {  // only this thread touches the segment's token count and slot ring
             const int g = a.gen[seg];
             int32_t *ring = a.slot_ring + (size_t)seg * (d + 1);

@@ -279,6 +279,46 @@ def test_decode_layer_range(api):
     assert torch.equal(a.cache.len, b.cache.len)
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", {}),
+    ("llava7b_b1", dict(L=3, H=8, N=200, T=3)),
+])
+def test_decode_without_append(api, name, kw):
+    """k_new = v_new = NULL: the query attends over the rows already cached and nothing changes."""
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 3) for b in range(w.B)])
+    budgets = [w.budget_rows()] * w.B
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    s.search(torch.tensor(budgets), scores=torch.from_numpy(scores).cuda())
+    s.compact(k, v)
+    qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
+    s.decode(qd, kn, vn)                           # one ordinary step first: the cache now ends in a decoded row
+    len1 = s.cache.len.clone()
+    ck, cv = s.cache.k.clone(), s.cache.v.clone()
+    q2, _, _ = wl.make_decode_inputs(w, 1, "cuda")
+    got = to_np32(s.decode(q2, None, None))
+    torch.cuda.synchronize()
+    bits = lambda t: t.view(torch.int16 if t.dtype == torch.bfloat16 else torch.int32)   # unused rows may hold NaN patterns
+    assert torch.equal(s.cache.len, len1)
+    assert torch.equal(bits(s.cache.k), bits(ck)) and torch.equal(bits(s.cache.v), bits(cv))
+    assert s.status.cpu().tolist() == [0] * w.B
+    offs = s.cache.row_offset.cpu().numpy()
+    worst = 0.0
+    for b in range(w.B):
+        for l in range(w.L):
+            seg = b * w.L + l
+            n, off = int(len1[seg]), int(offs[seg])
+            ref = oracle.decode_attn(to_np32(q2[b, l]), to_np32(ck[off:off + n]), to_np32(cv[off:off + n]),
+                                     float(scale[l]))
+            assert np.isfinite(got[b, l]).all()
+            worst = max(worst, float(np.abs(got[b, l] - ref).max()))
+    assert worst <= DECODE_TOL[w.dtype], worst
+    with pytest.raises(RuntimeError):              # one of the two alone is an argument error
+        s.decode(q2, kn, None)
+
+
 # --------------------------------------------------------------------------
 # importance score
 # --------------------------------------------------------------------------
