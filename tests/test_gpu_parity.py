@@ -217,6 +217,9 @@ def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
     ("llava7b_b16", dict(B=3, L=2, H=4, N=97, T=4)),
     ("tiny", dict(D=128, H=2, T=3)),
     ("llava7b_b1", dict(L=2, H=5, D=64, N=130, T=3)),
+    ("tiny", dict(D=128, H=32, L=2, N=100, T=3)),           # fp32 rows of 16 KiB: four-row units
+    ("llava7b_b1", dict(L=2, H=64, N=90, T=2)),              # 64 heads: four heads per consumer warp
+    ("llava7b_b1", dict(L=2, H=72, D=64, N=90, T=2)),        # more heads than the streaming kernel takes: two-kernel path
 ])
 def test_decode_matches_oracle(api, name, kw):
     w = wl.scaled(wl.WORKLOADS[name], **kw)
@@ -344,6 +347,28 @@ def test_score_matches_oracle(api, name, kw):
     # determinism: a second run gives the same bits
     again = s.score(q, k).cpu().numpy()
     np.testing.assert_array_equal(got, again)
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("llava7b_b1", dict(L=2, H=4, N=200)),           # bf16: tensor maps built from the strides
+    ("tiny", dict(N=90, H=3, L=2)),                  # fp32: strided loads
+])
+def test_score_token_major_layout(api, name, kw):
+    """Q and K stored [B, L, N, H, D] (one token's heads together, as a model's projections leave
+    them) and handed over through element strides: same scores, bit for bit, as the head-major copy."""
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
+    base = s.score(q, k).clone()
+    qt = q.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4)     # same values, token-major storage
+    kt = k.permute(0, 1, 3, 2, 4).contiguous().permute(0, 1, 3, 2, 4)
+    assert qt.stride(3) == w.H * w.D and qt.stride(2) == w.D and torch.equal(qt, q)
+    got = s.score(qt, kt)
+    assert torch.equal(got, base)
+    ref = oracle_scores(q, k, scale)
+    for (b, l), r in ref.items():
+        check_scores(got[b, l].cpu().numpy(), r, SCORE_TOL[w.dtype])
 
 
 def test_score_with_caller_lse(api):
