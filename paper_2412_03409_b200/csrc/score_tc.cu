@@ -135,16 +135,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64])
+// Both halves of a 128-column accumulator row: two loads in flight, one wait.
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, float (&v)[128])
 {
-    uint32_t r[64];
+    uint32_t r[64], q[64];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
         : "r"(taddr));
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(q[0]), "=r"(q[1]), "=r"(q[2]), "=r"(q[3]), "=r"(q[4]), "=r"(q[5]), "=r"(q[6]), "=r"(q[7]), "=r"(q[8]), "=r"(q[9]), "=r"(q[10]), "=r"(q[11]), "=r"(q[12]), "=r"(q[13]), "=r"(q[14]), "=r"(q[15]), "=r"(q[16]), "=r"(q[17]), "=r"(q[18]), "=r"(q[19]), "=r"(q[20]), "=r"(q[21]), "=r"(q[22]), "=r"(q[23]), "=r"(q[24]), "=r"(q[25]), "=r"(q[26]), "=r"(q[27]), "=r"(q[28]), "=r"(q[29]), "=r"(q[30]), "=r"(q[31]), "=r"(q[32]), "=r"(q[33]), "=r"(q[34]), "=r"(q[35]), "=r"(q[36]), "=r"(q[37]), "=r"(q[38]), "=r"(q[39]), "=r"(q[40]), "=r"(q[41]), "=r"(q[42]), "=r"(q[43]), "=r"(q[44]), "=r"(q[45]), "=r"(q[46]), "=r"(q[47]), "=r"(q[48]), "=r"(q[49]), "=r"(q[50]), "=r"(q[51]), "=r"(q[52]), "=r"(q[53]), "=r"(q[54]), "=r"(q[55]), "=r"(q[56]), "=r"(q[57]), "=r"(q[58]), "=r"(q[59]), "=r"(q[60]), "=r"(q[61]), "=r"(q[62]), "=r"(q[63])
+        : "r"(taddr + 64));
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 64; ++i) {
+        v[i] = __uint_as_float(r[i]);
+        v[64 + i] = __uint_as_float(q[i]);
+    }
 }
 // 2^x on the special-function unit, one instruction (inputs here are <= 0 or -inf; flushing
 // denormal results to zero is harmless for sums of probabilities).
@@ -376,18 +384,20 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // blocks 0..quarter in pass 1 (keys <= query), quarter..3 in pass 2 (queries >= key).
                 const int c_lo = (PASS == 2 && diag) ? quarter : 0;
                 const int c_hi = (PASS == 1 && diag) ? quarter : TT / 32 - 1;
+                bool released = false;
                 if (!diag) {
-                    // a full tile: two 64-column loads, so that the accumulator's read latency is paid
-                    // twice per tile
-#pragma unroll 1
-                    for (int half = 0; half < 2; ++half) {
-                        float v[64];
-                        tmem_ld64(taddr + half * 64, v);
-                        if (PASS == 1)
-                            lse_block<64>(v, sc, fast, run_max, run_sum);
-                        else
-                            col_sum += colsum_block<64>(v, &s_lse[rs.idx][half * 64], sc, false, lane);
-                    }
+                    // a full tile: the whole row comes into registers at once and the accumulator goes
+                    // back to the MMA thread before the arithmetic starts
+                    float v[128];
+                    tmem_ld128(taddr, v);
+                    fence_before();
+                    __syncwarp();
+                    if (lane == 0) bar_arrive(s_empty + rs.idx);
+                    released = true;
+                    if (PASS == 1)
+                        lse_block<128>(v, sc, fast, run_max, run_sum);
+                    else
+                        col_sum += colsum_block<128>(v, &s_lse[rs.idx][0], sc, false, lane);
                 } else {
 #pragma unroll 1
                     for (int cblk = c_lo; cblk <= c_hi; ++cblk) {
@@ -405,9 +415,11 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                     }
                 }
-                fence_before();
-                __syncwarp();
-                if (lane == 0) bar_arrive(s_empty + rs.idx);
+                if (!released) {
+                    fence_before();
+                    __syncwarp();
+                    if (lane == 0) bar_arrive(s_empty + rs.idx);
+                }
                 rs.next(2);
             }
             if (PASS == 1) {
