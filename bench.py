@@ -344,8 +344,9 @@ def run_ours(args):
     if e2e is not None:
         line["e2e"] = {"value": world * w.B * w.T / (e2e["ms"] * 1e-3), "unit": "tok/s",
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                       "note": "host pinned Q,K,V and per-token q,k,v copied in, outputs copied out, "
-                               "wall clock, no L2 flush"}
+                       "note": "host pinned Q,K,V and per-token q,k,v copied in, outputs copied out and "
+                               "synchronised per token; the next prompt uploads on a copy stream while "
+                               "this one decodes; wall clock over the steps, no L2 flush"}
     if world == 1 and not args.no_cpu_baseline:
         v_cpu, desc, spent = time_oracle_sample(w, score_layers=min(w.L, 16), decode_steps=(0, 1, 2, 3))
         line["cpu_baseline"] = {"value": v_cpu, "unit": "tok/s", "cores": 1, "kind": "oracle",
@@ -362,35 +363,53 @@ def LAUNCHES_PER_STEP(w):
 
 
 def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):
-    """Same path with host buffers: inputs start in pinned host memory every step and
-    every decode output is read back."""
+    """Same path with host buffers: every step's prompt tensors start in pinned host memory and every
+    token's q, k, v are copied in and its output copied out, with a host synchronisation per token
+    (the result is needed before the next token).  The way a serving loop would run it: the next
+    prompt's upload goes through a copy stream into a second set of device buffers while the
+    current prompt decodes; a token's three inputs travel as one copy."""
     hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
-    hpool = [tuple(x.cpu().pin_memory() for x in p) for p in pool]
-    dq, dk, dv = (torch.empty_like(t) for t in (q, k, v))
-    dd = [torch.empty_like(x) for x in pool[0]]
+    hpool = [torch.stack([x.cpu() for x in p]).pin_memory() for p in pool]      # [3, B, L, H, D] per token
+    dbuf = [tuple(torch.empty_like(t) for t in (q, k, v)) for _ in range(2)]
+    dtok = torch.empty_like(hpool[0], device=dev)
     hout = torch.empty(s.out.shape, dtype=s.out.dtype).pin_memory()
-    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv)) + \
-        w.T * sum(x.numel() * x.element_size() for x in hpool[0])
+    h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv)) + w.T * hpool[0].numel() * hpool[0].element_size()
     d2h = w.T * hout.numel() * hout.element_size()
+    main = torch.cuda.current_stream()
+    copy = torch.cuda.Stream(device=dev)
+    ready = [torch.cuda.Event() for _ in range(2)]
+    free = [torch.cuda.Event() for _ in range(2)]
 
-    def one():
-        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
-        s.score(dq, dk)
-        s.search(None, tol=w.tol)
-        s.compact(dk, dv)
-        for t in range(w.T):
-            hp = hpool[t % len(hpool)]
-            for d_, h_ in zip(dd, hp):
+    def upload(i):
+        with torch.cuda.stream(copy):
+            copy.wait_event(free[i % 2])            # the buffers' previous prompt has been compacted
+            for d_, h_ in zip(dbuf[i % 2], (hq, hk, hv)):
                 d_.copy_(h_, non_blocking=True)
-            s.decode(dd[0], dd[1], dd[2])
-            hout.copy_(s.out, non_blocking=True)
-            torch.cuda.synchronize()          # the token's result is needed on the host
+            ready[i % 2].record(copy)
 
-    one()
+    def run(n):
+        for e in free:
+            e.record(main)
+        upload(0)
+        for i in range(n):
+            if i + 1 < n:
+                upload(i + 1)
+            dq, dk, dv = dbuf[i % 2]
+            main.wait_event(ready[i % 2])
+            s.score(dq, dk)
+            s.search(None, tol=w.tol)
+            s.compact(dk, dv)
+            free[i % 2].record(main)
+            for t in range(w.T):
+                dtok.copy_(hpool[t % len(hpool)], non_blocking=True)
+                s.decode(dtok[0], dtok[1], dtok[2])
+                hout.copy_(s.out, non_blocking=True)
+                main.synchronize()                # the token's result is needed on the host
+
+    run(1)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
-    for _ in range(steps):
-        one()
+    run(steps)
     torch.cuda.synchronize()
     return {"ms": 1e3 * (time.perf_counter() - t0) / steps, "h2d": h2d, "d2h": d2h}
 
