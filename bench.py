@@ -53,8 +53,8 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
-# DRAM bytes (read + write) of one decode_stream_kernel launch from the ncu capture summarised in
-# profiles/decode_stream_kernel_<workload>.md, keyed by workload, with the hash of the kernel source
+# DRAM bytes (read + write) of one decode_stream_kernel launch from an ncu capture (its summary is
+# kept under profiles/), keyed by workload, with the hash of the kernel source
 # the counters were taken on: once that file changes the figure is stale and `traffic` reads null.
 DECODE_TRAFFIC = {"llava7b_b1": (103.50e6, "720ee5e8ea2b1990")}
 
