@@ -745,6 +745,93 @@ __global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_kernel(const 
     }
 }
 
+// Merge kernel for few segments: one warp per (active segment, head), no shared memory, no block
+// barrier.  The segment's record is read twice: before griddepcontrol.wait (the stream kernel wrote
+// it in its first microsecond, so this early copy is almost always the final one), so that the
+// loads of the partials can go out the moment the wait returns, and again after it, in flight
+// together with those loads.  The early copy's result is kept only if the two copies agree;
+// otherwise the merge is redone from the second.  The early copy is never trusted for addresses
+// beyond the slots that exist, nor for what is written to len.
+template <typename T, int D>
+__global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_small_kernel(const DecodeArgs a, int nslots)
+{
+    constexpr int kSlotStride = D + 4, EPM = D / 32, KB = 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int item = blockIdx.x * kFinishWarps + warp;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // e.g. the next decode step
+    if (item >= a.nact * a.H) return;
+    const int si = item / a.H, h = item - si * a.H;
+    const int4 *recp = reinterpret_cast<const int4 *>(a.plan) + si;
+    const int4 early = __ldcg(recp);
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream kernel's writes are visible
+    const int4 late = __ldcg(recp);
+    const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+    const size_t cstride = (size_t)a.H * kSlotStride;
+
+    int4 r = early;
+    float M = -INFINITY, z = 0.f, o[EPM];
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        M = -INFINITY;
+        z = 0.f;
+#pragma unroll
+        for (int i = 0; i < EPM; ++i) o[i] = 0.f;
+        const bool usable = r.x >= 0 && r.y >= 0 && r.z > 1 && r.y + si + r.z <= nslots;
+        if (usable) {
+            const int c_first = r.y, ncontrib = r.z;
+            const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;
+#pragma unroll 1
+            for (int k0 = 0; k0 < ncontrib; k0 += KB) {
+                float2 ml[KB];
+                float x[KB][EPM];
+#pragma unroll
+                for (int kk = 0; kk < KB; ++kk) {
+                    const float *sl = base + (size_t)min(k0 + kk, ncontrib - 1) * cstride;
+                    ml[kk] = __ldcg(reinterpret_cast<const float2 *>(sl + D));
+                    LoadF<EPM>::ld(sl + lane * EPM, x[kk]);
+                }
+                float mb = M;
+#pragma unroll
+                for (int kk = 0; kk < KB; ++kk)
+                    if (k0 + kk < ncontrib) mb = fmaxf(mb, ml[kk].x);
+                const float corr = M == -INFINITY ? 0.f : exp2f(M - mb);
+                z *= corr;
+#pragma unroll
+                for (int i = 0; i < EPM; ++i) o[i] *= corr;
+                M = mb;
+#pragma unroll
+                for (int kk = 0; kk < KB; ++kk) {
+                    if (k0 + kk < ncontrib) {
+                        const float ww = exp2f(ml[kk].x - mb);
+                        z = fmaf(ww, ml[kk].y, z);
+#pragma unroll
+                        for (int i = 0; i < EPM; ++i) o[i] = fmaf(ww, x[kk][i], o[i]);
+                    }
+                }
+            }
+        }
+        if (attempt == 1 || (late.x == r.x && late.y == r.y && late.z == r.z && late.w == r.w)) break;
+        r = late;
+    }
+    // from here on r is the record as the finished stream kernel left it
+    if (r.x < 0) return;  // could not take a row: reported and zero-filled by the stream kernel
+    if (h == 0 && lane == 0) {
+        a.len[seg] = r.x;
+        const int d = a.k_new ? a.evict_distance : 0;
+        if (d > 0) {  // only this thread touches the segment's token count and slot ring
+            const int g = a.gen[seg];
+            int32_t *ring = a.slot_ring + (size_t)seg * (d + 1);
+            if (r.w >> 30) ring[(g - d) % (d + 1)] = -1;  // the token d steps back gave up its slot
+            ring[g % (d + 1)] = r.w & 0x3fffffff;
+            a.gen[seg] = g + 1;
+        }
+    }
+    if (r.z <= 1) return;  // one CTA covered the segment and wrote its output
+    const float inv = 1.f / z;
+#pragma unroll
+    for (int i = 0; i < EPM; ++i) o[i] *= inv;
+    Pack<T, EPM>::store(reinterpret_cast<T *>(a.out) + ((size_t)seg * a.H + h) * D + lane * EPM, o);
+}
+
 static size_t plan_bytes(int nact) { return round_up((size_t)nact * sizeof(int4), kWsAlign); }
 
 size_t decode_stream_ws_bytes(const pkv_shape *s)
@@ -793,10 +880,15 @@ static int launch_variant(const DecodeArgs &a, int sms, cudaStream_t st)
     cfg.gridDim = dim3(blocks < sms ? blocks : sms);
     cfg.blockDim = dim3(kFinishWarps * 32);
     cfg.dynamicSmemBytes = 0;
-    if (hg == 2)
+    if (hg == 2) {
         e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D, 2>, a);
-    else
+    } else if (items <= sms * kFinishWarps) {  // a warp for every (segment, head): the barrier-free kernel
+        cfg.gridDim = dim3(blocks);
+        const int nslots = 256 + a.nseg_total;  // partial slots the workspace holds
+        e = cudaLaunchKernelEx(&cfg, decode_finish_small_kernel<T, D>, a, nslots);
+    } else {
         e = cudaLaunchKernelEx(&cfg, decode_finish_kernel<T, D, 1>, a);
+    }
     if (e != cudaSuccess) {
         set_cuda_error(e, "decode_finish_kernel");
         return PKV_ERR_CUDA;
