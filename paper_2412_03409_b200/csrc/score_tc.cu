@@ -36,6 +36,7 @@ struct ScoreArgs {
     float *lse2;     // [B*L*H][Npad] log2-sum-exp of scaled logits, +inf beyond N
     float *partial;  // [B*L*H][N] per-head column sums
     int32_t *abort_word;  // device word set when a bounded wait runs out (may be null)
+    int *next_item;       // [2] work counters, one per pass; zeroed before the first pass is launched
     int L, H, N, Npad, tiles, nseg;
 };
 
@@ -135,6 +136,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&v)[64])
+{
+    uint32_t r[64];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]), "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]), "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]), "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]), "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 64; ++i) v[i] = __uint_as_float(r[i]);
+}
 // Both halves of a 128-column accumulator row: two loads in flight, one wait.
 __device__ __forceinline__ void tmem_ld128(uint32_t taddr, float (&v)[128])
 {
@@ -227,18 +239,20 @@ __device__ __forceinline__ float colsum_block(const float (&v)[NC], const float 
     return (p4[0] + p4[1]) + (p4[2] + p4[3]);
 }
 
-// Work item w -> (segment-head sh, tile t).  The tiles of one head are consecutive items, so
-// the CTAs running at any moment share a few dozen heads whose Q and K stay in L2 and every
-// operand byte comes from HBM once per pass.  Pass 2 walks the heads backwards: it starts on
-// what pass 1 touched last.  A CTA's successive items (stride gridDim.x, chosen by the launcher to
-// share no factor with the tiles per head) cycle through the tile index, which mixes long and
-// short items evenly.
+// Work item w -> (segment-head sh, tile t).  CTAs take items in order from a counter.  The tiles
+// of one head are consecutive items, so the CTAs running at any moment share a few dozen heads
+// whose Q and K stay in L2 and every operand byte comes from HBM once per pass; within a head
+// the longest item comes first (pass 1: the last query tile, pass 2: the first key tile), so
+// that what is left for the end of the pass is short.  Pass 2 walks the heads backwards: it
+// starts on what pass 1 touched last.
 template <int PASS> __device__ __forceinline__ void decode_item(int w, int nsh, int tiles, int &sh, int &t)
 {
-    const int q = w / tiles;
-    t = w - q * tiles;
+    const int q = w / tiles, r = w - q * tiles;
+    t = PASS == 1 ? tiles - 1 - r : r;
     sh = PASS == 1 ? q : nsh - 1 - q;
 }
+
+constexpr int kItemQ = 4;  // item numbers in flight between the loader and the other roles
 
 // PASS 1: stationary = Q tile t, streamed = K tiles 0..t.  PASS 2: stationary = K tile t,
 // streamed = Q tiles t..tiles-1.
@@ -257,8 +271,10 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     uint64_t *bars = reinterpret_cast<uint64_t *>(sB + kStagesB * TILE);
     uint64_t *a_full = bars, *a_empty = bars + 1, *b_full = bars + 2, *b_empty = b_full + kStagesB;
     uint64_t *s_full = b_empty + kStagesB, *s_empty = s_full + 2;
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(s_empty + 2);
+    uint64_t *q_full = s_empty + 2, *q_empty = q_full + kItemQ;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_empty + kItemQ);
     __shared__ int s_abort;
+    __shared__ int q_item[kItemQ];  // the loader's announcements: an item number, or -1 for the end
     __shared__ __align__(16) float s_lse[2][TT];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -279,6 +295,10 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             bar_init(s_full + i, 1);
             bar_init(s_empty + i, 4);
         }
+        for (int i = 0; i < kItemQ; ++i) {
+            bar_init(q_full + i, 1);
+            bar_init(q_empty + i, 5);  // the MMA thread and the four reader warps
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {  // two 128-column fp32 accumulators
@@ -297,8 +317,18 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (lane == 0) {
             bool dead = false;
             uint32_t a_phase = 0;
-            Ring2 rb{0, 0u};
-            for (int w = blockIdx.x; w < nitems && !dead; w += gridDim.x) {
+            Ring2 rb{0, 0u}, rq{0, 0u};
+            int *ctr = a.next_item + (PASS - 1);
+            int next = atomicAdd(ctr, 1);  // asked for one item ahead: the answer takes a microsecond
+            for (;;) {
+                const int w = next < nitems ? next : -1;
+                if (w >= 0) next = atomicAdd(ctr, 1);
+                bar_wait(q_empty + rq.idx, rq.phase ^ 1u, dead, &s_abort);
+                if (dead) break;
+                q_item[rq.idx] = w;
+                bar_arrive(q_full + rq.idx);
+                rq.next(kItemQ);
+                if (w < 0) break;
                 int sh, t;
                 decode_item<PASS>(w, nsh, a.tiles, sh, t);
                 const int seg = sh / a.H, h = sh - seg * a.H, b = seg / a.L, l = seg - b * a.L;
@@ -326,8 +356,14 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (lane == 0) {
             bool dead = false;
             uint32_t a_phase = 0;
-            Ring2 rb{0, 0u}, rs{0, 0u};
-            for (int w = blockIdx.x; w < nitems && !dead; w += gridDim.x) {
+            Ring2 rb{0, 0u}, rs{0, 0u}, rq{0, 0u};
+            for (;;) {
+                bar_wait(q_full + rq.idx, rq.phase, dead, &s_abort);
+                if (dead) break;
+                const int w = q_item[rq.idx];
+                bar_arrive(q_empty + rq.idx);
+                rq.next(kItemQ);
+                if (w < 0) break;
                 int sh, t;
                 decode_item<PASS>(w, nsh, a.tiles, sh, t);
                 bar_wait(a_full, a_phase, dead, &s_abort);
@@ -359,8 +395,15 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int row = quarter * 32 + lane;
         const int rtid = tid - 64;  // 0..127 among the reader warps
         bool dead = false;
-        Ring2 rs{0, 0u};
-        for (int w = blockIdx.x; w < nitems; w += gridDim.x) {
+        Ring2 rs{0, 0u}, rq{0, 0u};
+        for (;;) {
+            bar_wait(q_full + rq.idx, rq.phase, dead, &s_abort);
+            if (dead) break;
+            const int w = q_item[rq.idx];
+            __syncwarp();
+            if (lane == 0) bar_arrive(q_empty + rq.idx);
+            rq.next(kItemQ);
+            if (w < 0) break;
             int sh, t;
             decode_item<PASS>(w, nsh, a.tiles, sh, t);
             const int seg = sh / a.H, l = seg % a.L;
@@ -388,16 +431,28 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (!diag) {
                     // a full tile: the whole row comes into registers at once and the accumulator goes
                     // back to the MMA thread before the arithmetic starts
-                    float v[128];
-                    tmem_ld128(taddr, v);
-                    fence_before();
-                    __syncwarp();
-                    if (lane == 0) bar_arrive(s_empty + rs.idx);
-                    released = true;
-                    if (PASS == 1)
+                    if (PASS == 1) {
+                        float v[128];
+                        tmem_ld128(taddr, v);
+                        fence_before();
+                        __syncwarp();
+                        if (lane == 0) bar_arrive(s_empty + rs.idx);
+                        released = true;
                         lse_block<128>(v, sc, fast, run_max, run_sum);
-                    else
-                        col_sum += colsum_block<128>(v, &s_lse[rs.idx][0], sc, false, lane);
+                    } else {  // (pass 2 keeps more state: half a row at a time fits its registers)
+#pragma unroll 1
+                        for (int half = 0; half < 2; ++half) {
+                            float v[64];
+                            tmem_ld64(taddr + half * 64, v);
+                            if (half == 1) {
+                                fence_before();
+                                __syncwarp();
+                                if (lane == 0) bar_arrive(s_empty + rs.idx);
+                                released = true;
+                            }
+                            col_sum += colsum_block<64>(v, &s_lse[rs.idx][half * 64], sc, false, lane);
+                        }
+                    }
                 } else {
 #pragma unroll 1
                     for (int cblk = c_lo; cblk <= c_hi; ++cblk) {
@@ -502,15 +557,10 @@ int launch_pass(const CUtensorMap &mq, const CUtensorMap &mk, const ScoreArgs &a
     int rc = ensure_dynamic_smem((const void *)score_tile_kernel<PASS, D>, (int)smem, done);
     if (rc != PKV_OK) return rc;
     const int items = a.nseg * a.H * a.tiles;
-    // A CTA takes items blockIdx.x, + grid, + 2 grid, ...: with a grid size that shares no factor
-    // with the tiles per head its items run through every tile index (long and short items) evenly.
-    // (296 CTAs and 16 tiles share 8: every CTA would see two tile indices only, and the slowest
-    // would do 12 tiles per item against a mean of 8.5.)
-    int grid = items < 2 * sms ? items : 2 * sms;
-    if (items > grid) {
-        auto gcd = [](int x, int y) { while (y) { int r = x % y; x = y; y = r; } return x; };
-        while (grid > sms && gcd(grid, a.tiles) != 1) --grid;
-    }
+    // CTAs take items from a counter as they finish (long and short items mix in any case; with a
+    // fixed stride, 296 CTAs and 16 tiles per head left every CTA two tile indices only, and the
+    // slowest did 12 tiles per item against a mean of 8.5).
+    const int grid = items < 2 * sms ? items : 2 * sms;
     score_tile_kernel<PASS, D><<<grid, 192, smem, st>>>(mq, mk, a);
     return check_launch(PASS == 1 ? "score_tile_kernel<1>" : "score_tile_kernel<2>");
 }
@@ -528,7 +578,8 @@ size_t score_tc_ws_bytes(const pkv_shape *s)
 {
     const size_t rows = (size_t)s->batch * s->layers * s->heads;
     const size_t npad = ((size_t)s->prompt_len + TT - 1) / TT * TT;
-    return round_up(rows * s->prompt_len * sizeof(float), kWsAlign) + round_up(rows * npad * sizeof(float), kWsAlign);
+    return round_up(rows * s->prompt_len * sizeof(float), kWsAlign) + round_up(rows * npad * sizeof(float), kWsAlign) +
+           kWsAlign;  // the two work counters
 }
 
 // Returns PKV_OK, an error, or -1 when the tensor maps cannot describe the caller's layout.
@@ -547,6 +598,14 @@ int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const voi
     a.L = L; a.H = H; a.N = N;
     a.tiles = (N + TT - 1) / TT;
     a.Npad = a.tiles * TT;
+    a.next_item = (int *)((unsigned char *)a.lse2 + round_up(rows * a.Npad * sizeof(float), kWsAlign));
+    {
+        cudaError_t e = cudaMemsetAsync(a.next_item, 0, 2 * sizeof(int), st);
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "cudaMemsetAsync(score work counters)");
+            return PKV_ERR_CUDA;
+        }
+    }
     a.nseg = B * L;
 
     static int sm_count[64] = {};
