@@ -14,9 +14,11 @@
 // Roles per CTA (192 threads): warp 0 lane 0 issues TMA, warp 1 owns tensor memory and its
 // lane 0 issues the MMAs, warps 2-5 read the accumulator (tcgen05.ld, one TMEM lane quarter
 // per warp) and do the exponentials.  Two accumulators alternate so that the MMAs of tile
-// j + 1 overlap the exponentials of tile j; two CTAs share an SM.  Every mbarrier wait is
-// bounded: when one runs out the CTA stops waiting, reports PKV_DEV_TIMEOUT and still
-// releases its tensor memory.
+// j + 1 overlap the exponentials of tile j; two CTAs share an SM.  Work items (one stationary
+// tile and the tiles streamed against it) come from a device counter: the TMA thread takes the
+// next number and announces it to the other roles through a four-entry shared-memory queue,
+// so CTAs that run faster do more.  Every mbarrier wait is bounded: when one runs out the CTA
+// stops waiting, reports PKV_DEV_TIMEOUT and still releases its tensor memory.
 #include <cuda.h>
 
 #include "common.cuh"
