@@ -95,6 +95,8 @@ const char *prefixkv_last_cuda_error(void);
  *               NULL the library computes it in a first pass
  *   scores      [B,L,N] fp32, out
  * bf16 inputs use tensor cores with fp32 accumulation; fp32 inputs use fp32 FMA.
+ * The workspace holds per-head partial sums and work counters: calls that share one must
+ * not overlap on the GPU.
  */
 int prefixkv_score(const pkv_shape *shape, const void *q, pkv_strides qs, const void *k,
                    pkv_strides ks, const float *layer_scale, const float *lse, float *scores,
