@@ -282,6 +282,33 @@ def test_decode_layer_range(api):
     assert torch.equal(a.cache.len, b.cache.len)
 
 
+def test_decode_empty_segment_is_reported(api):
+    """A segment with no rows (never compacted) cannot be attended over: the sample's status says
+    so, its output is zero, its length stays, and the other segments are unaffected."""
+    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], B=2, L=3, H=4, N=80, T=2)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 11) for b in range(w.B)])
+    a = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    b = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    for s in (a, b):
+        s.search(w.budget_rows(), scores=torch.from_numpy(scores).cuda())
+        s.compact(k, v)
+    empty = 1 * w.L + 2                              # sample 1, layer 2
+    b.cache.len[empty] = 0
+    qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
+    ref = a.decode(qd, kn, vn).float().clone()
+    got = b.decode(qd, kn, vn).float()
+    torch.cuda.synchronize()
+    assert b.status.cpu().tolist() == [0, api.DEV_CAPACITY]
+    assert int(b.cache.len[empty]) == 0
+    assert (got[1, 2] == 0).all()
+    mask = torch.ones(w.B, w.L, dtype=torch.bool)
+    mask[1, 2] = False
+    assert torch.equal(got[mask.cuda()], ref[mask.cuda()])
+    assert torch.equal(b.cache.len[mask.flatten().cuda()], a.cache.len[mask.flatten().cuda()])
+
+
 @pytest.mark.parametrize("name,kw", [
     ("tiny", {}),
     ("llava7b_b1", dict(L=3, H=8, N=200, T=3)),
