@@ -946,7 +946,9 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     const bool bf = s->dtype == PKV_BF16;
     const int vec_per_head = D / (int)(16 / es);
     // (lanes per row, heads per warp): at most 17 warps, and few enough registers of per-head
-    // state that each SM sub-partition's register file holds its warps.
+    // state that each SM sub-partition's register file holds its warps.  (The last template
+    // argument is the block-size bound a variant is compiled for: 9, 12 or 17 warps, the smaller
+    // ones with room for more registers per thread.)
     int lpr = 8, hpw = H <= 16 ? 1 : (H <= 32 ? 2 : 4);
     if (H > 16 && vec_per_head >= 16) lpr = 16;
     if (vec_per_head < lpr || H % hpw != 0) return -1;
@@ -958,17 +960,21 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     PKV_V(T, DD, 8, 1, 8, 544);  \
     PKV_V(T, DD, 8, 2, 8, 544);  \
     PKV_V(T, DD, 8, 4, 8, 288);  \
+    PKV_V(T, DD, 8, 4, 8, 384);  \
     PKV_V(T, DD, 8, 4, 8, 544);  \
     PKV_V(T, DD, 8, 1, 4, 544);  \
     PKV_V(T, DD, 8, 2, 4, 544);  \
     PKV_V(T, DD, 8, 4, 4, 288);  \
+    PKV_V(T, DD, 8, 4, 4, 384);  \
     PKV_V(T, DD, 8, 4, 4, 544)
 #define PKV_WIDE(T, DD)           \
     PKV_V(T, DD, 16, 2, 8, 544);  \
     PKV_V(T, DD, 16, 4, 8, 288);  \
+    PKV_V(T, DD, 16, 4, 8, 384);  \
     PKV_V(T, DD, 16, 4, 8, 544);  \
     PKV_V(T, DD, 16, 2, 4, 544);  \
     PKV_V(T, DD, 16, 4, 4, 288);  \
+    PKV_V(T, DD, 16, 4, 4, 384);  \
     PKV_V(T, DD, 16, 4, 4, 544)
     if (bf && D == 128) {
         PKV_FAMILY(__nv_bfloat16, 128);
