@@ -956,40 +956,43 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
 #define PKV_V(T, DD, LPR, HPW, UR, MAXT)                                       \
     if (lpr == LPR && hpw == HPW && ur == UR && (a.nwarps + 1) * 32 <= MAXT) \
         return launch_variant<T, DD, LPR, HPW, UR, MAXT>(a, sms, st)
-#define PKV_FAMILY(T, DD)        \
-    PKV_V(T, DD, 8, 1, 8, 544);  \
-    PKV_V(T, DD, 8, 2, 8, 544);  \
-    PKV_V(T, DD, 8, 4, 8, 288);  \
-    PKV_V(T, DD, 8, 4, 8, 384);  \
-    PKV_V(T, DD, 8, 4, 8, 544);  \
-    PKV_V(T, DD, 8, 1, 4, 544);  \
-    PKV_V(T, DD, 8, 2, 4, 544);  \
-    PKV_V(T, DD, 8, 4, 4, 288);  \
-    PKV_V(T, DD, 8, 4, 4, 384);  \
+    // Only what the choice above can ask for is instantiated: eight lanes per row with one head per
+    // warp (at most 16 heads) for every type; with more heads per warp only where a head row has
+    // fewer than sixteen 16-byte vectors (bf16, D = 64); sixteen lanes per row otherwise.  Four
+    // heads per warp means more than 32 heads, i.e. at least ten warps.
+#define PKV_NARROW1(T, DD)      \
+    PKV_V(T, DD, 8, 1, 8, 544); \
+    PKV_V(T, DD, 8, 1, 4, 544)
+#define PKV_NARROW(T, DD)       \
+    PKV_V(T, DD, 8, 2, 8, 544); \
+    PKV_V(T, DD, 8, 4, 8, 384); \
+    PKV_V(T, DD, 8, 4, 8, 544); \
+    PKV_V(T, DD, 8, 2, 4, 544); \
+    PKV_V(T, DD, 8, 4, 4, 384); \
     PKV_V(T, DD, 8, 4, 4, 544)
-#define PKV_WIDE(T, DD)           \
-    PKV_V(T, DD, 16, 2, 8, 544);  \
-    PKV_V(T, DD, 16, 4, 8, 288);  \
-    PKV_V(T, DD, 16, 4, 8, 384);  \
-    PKV_V(T, DD, 16, 4, 8, 544);  \
-    PKV_V(T, DD, 16, 2, 4, 544);  \
-    PKV_V(T, DD, 16, 4, 4, 288);  \
-    PKV_V(T, DD, 16, 4, 4, 384);  \
+#define PKV_WIDE(T, DD)          \
+    PKV_V(T, DD, 16, 2, 8, 544); \
+    PKV_V(T, DD, 16, 4, 8, 384); \
+    PKV_V(T, DD, 16, 4, 8, 544); \
+    PKV_V(T, DD, 16, 2, 4, 544); \
+    PKV_V(T, DD, 16, 4, 4, 384); \
     PKV_V(T, DD, 16, 4, 4, 544)
     if (bf && D == 128) {
-        PKV_FAMILY(__nv_bfloat16, 128);
+        PKV_NARROW1(__nv_bfloat16, 128);
         PKV_WIDE(__nv_bfloat16, 128);
     } else if (bf && D == 64) {
-        PKV_FAMILY(__nv_bfloat16, 64);
+        PKV_NARROW1(__nv_bfloat16, 64);
+        PKV_NARROW(__nv_bfloat16, 64);
     } else if (!bf && D == 128) {
-        PKV_FAMILY(float, 128);
+        PKV_NARROW1(float, 128);
         PKV_WIDE(float, 128);
     } else if (!bf && D == 64) {
-        PKV_FAMILY(float, 64);
+        PKV_NARROW1(float, 64);
         PKV_WIDE(float, 64);
     }
+#undef PKV_NARROW1
+#undef PKV_NARROW
 #undef PKV_WIDE
-#undef PKV_FAMILY
 #undef PKV_V
     return -1;
 }
