@@ -221,8 +221,18 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
     if (!ws || !aligned(ws, kWsAlign) || ws_bytes < decode_ws_bytes(shape)) return PKV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     {
-        int rc = launch_decode_stream(shape, cache, q, k_new, v_new, layer_scale, layer_begin,
-                                      layer_end, out, dev_status, ws, st);
+        // The streaming kernel plans at most 1024 segments at a time: a larger batch x layer range
+        // goes through it in layer chunks, one launch after the other on the stream.
+        const int max_active = 1024;
+        int step = layer_end - layer_begin;
+        if ((size_t)shape->batch * step > (size_t)max_active && shape->batch <= max_active)
+            step = max_active / shape->batch;
+        int rc = -1;
+        for (int lb = layer_begin; lb < layer_end; lb += step) {
+            const int le = lb + step < layer_end ? lb + step : layer_end;
+            rc = launch_decode_stream(shape, cache, q, k_new, v_new, layer_scale, lb, le, out, dev_status, ws, st);
+            if (rc != PKV_OK) break;
+        }
         if (rc >= 0) return rc;  // -1: shape outside the streaming kernel, use the two-kernel path
     }
     if (cache->evict_distance != 0) return PKV_ERR_UNSUPPORTED;  // pruning lives in the streaming kernel

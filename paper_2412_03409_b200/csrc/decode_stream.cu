@@ -775,7 +775,10 @@ __global__ void __launch_bounds__(kFinishWarps * 32) decode_finish_small_kernel(
         z = 0.f;
 #pragma unroll
         for (int i = 0; i < EPM; ++i) o[i] = 0.f;
-        const bool usable = r.x >= 0 && r.y >= 0 && r.z > 1 && r.y + si + r.z <= nslots;
+        // (the early copy may be anything, e.g. what another shape's call left in the workspace:
+        // bound each field before adding them, so that the sum cannot wrap)
+        const bool usable = r.x >= 0 && r.y >= 0 && r.y < nslots && r.z > 1 && r.z <= nslots &&
+                            r.y + si + r.z <= nslots;
         if (usable) {
             const int c_first = r.y, ncontrib = r.z;
             const float *base = a.scratch + ((size_t)(c_first + si) * a.H + h) * kSlotStride;

@@ -220,6 +220,7 @@ def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
     ("tiny", dict(D=128, H=32, L=2, N=100, T=3)),           # fp32 rows of 16 KiB: four-row units
     ("llava7b_b1", dict(L=2, H=64, N=90, T=2)),              # 64 heads: four heads per consumer warp
     ("llava7b_b1", dict(L=2, H=72, D=64, N=90, T=2)),        # more heads than the streaming kernel takes: two-kernel path
+    ("llava7b_b16", dict(B=40, L=32, H=2, D=64, N=24, T=2)),  # 1280 segments: two layer chunks through the streaming kernel
 ])
 def test_decode_matches_oracle(api, name, kw):
     w = wl.scaled(wl.WORKLOADS[name], **kw)
@@ -280,6 +281,32 @@ def test_decode_layer_range(api):
         b.decode(qd, kn, vn, layer_begin=l, layer_end=l + 1)
     assert (full - b.out.float()).abs().max() <= DECODE_TOL[w.dtype]
     assert torch.equal(a.cache.len, b.cache.len)
+
+
+@pytest.mark.parametrize("byte", [0x7f, 0xff, 0x00])
+def test_decode_with_stale_workspace(api, byte):
+    """The decode workspace may hold anything (another shape's partials, an earlier call's plan):
+    results do not depend on it.  (The merge kernel looks at its plan record early, before the record
+    is final, and must bound what it does with that copy.)"""
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=6, H=8, N=300, T=2)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = torch.from_numpy(wl.synthetic_scores(w.L, w.N, 5)[None]).cuda()
+    a = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    b = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
+    for s in (a, b):
+        s.search(w.budget_rows(), scores=scores)
+        s.compact(k, v)
+    b.ws_decode.fill_(byte)
+    for t in range(w.T):
+        qd, kn, vn = wl.make_decode_inputs(w, t, "cuda")
+        ref = a.decode(qd, kn, vn).clone()
+        got = b.decode(qd, kn, vn)
+        torch.cuda.synchronize()
+        assert torch.equal(got, ref)
+        b.ws_decode[: 4096].fill_(byte)            # and again over the plan records of the call just made
+    assert torch.equal(a.cache.len, b.cache.len)
+    assert a.status.cpu().tolist() == b.status.cpu().tolist() == [0]
 
 
 def test_decode_empty_segment_is_reported(api):
