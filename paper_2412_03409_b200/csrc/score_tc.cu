@@ -416,9 +416,13 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             float run_max = -INFINITY, run_sum = 0.f;  // pass 1
             float col_sum = 0.f;                       // pass 2
             const int j0 = PASS == 1 ? 0 : t, j1 = PASS == 1 ? t : a.tiles - 1;
+            // pass 2: a tile's 128 query normalisers are shared by all readers through shared memory;
+            // each thread fetches its one a tile ahead, so that the load's latency is not in the way
+            float lse_mine = PASS == 2 ? __ldg(lse_row + j0 * TT + rtid) : 0.f;
             for (int j = j0; j <= j1; ++j) {
-                if (PASS == 2) {  // this tile's 128 query normalisers, shared by all readers
-                    s_lse[rs.idx][rtid] = __ldg(lse_row + j * TT + rtid);
+                if (PASS == 2) {
+                    s_lse[rs.idx][rtid] = lse_mine;
+                    if (j < j1) lse_mine = __ldg(lse_row + (j + 1) * TT + rtid);
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                 }
                 bar_wait(s_full + rs.idx, rs.phase, dead, &s_abort);
