@@ -277,7 +277,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(q_empty + kItemQ);
     __shared__ int s_abort;
     __shared__ int q_item[kItemQ];  // the loader's announcements: an item number, or -1 for the end
-    __shared__ __align__(16) float s_lse[2][TT];
+    __shared__ __align__(16) float s_lse[2][4][TT];  // [accumulator][reader warp][query of the tile]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const CUtensorMap *map_stat = PASS == 1 ? &map_q : &map_k;
@@ -395,7 +395,6 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---- accumulator readers: one TMEM lane (tile row) per thread ----------------------------
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
-        const int rtid = tid - 64;  // 0..127 among the reader warps
         bool dead = false;
         Ring2 rs{0, 0u}, rq{0, 0u};
         for (;;) {
@@ -416,14 +415,17 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             float run_max = -INFINITY, run_sum = 0.f;  // pass 1
             float col_sum = 0.f;                       // pass 2
             const int j0 = PASS == 1 ? 0 : t, j1 = PASS == 1 ? t : a.tiles - 1;
-            // pass 2: a tile's 128 query normalisers are shared by all readers through shared memory;
-            // each thread fetches its one a tile ahead, so that the load's latency is not in the way
-            float lse_mine = PASS == 2 ? __ldg(lse_row + j0 * TT + rtid) : 0.f;
+            // pass 2: every thread needs the tile's 128 query normalisers.  Each warp keeps its own copy
+            // in shared memory (four per lane, fetched a tile ahead so that the load's latency is not
+            // in the way), so the reader warps never wait for one another.
+            float4 lse_mine = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (PASS == 2) lse_mine = __ldg(reinterpret_cast<const float4 *>(lse_row + j0 * TT) + lane);
             for (int j = j0; j <= j1; ++j) {
                 if (PASS == 2) {
-                    s_lse[rs.idx][rtid] = lse_mine;
-                    if (j < j1) lse_mine = __ldg(lse_row + (j + 1) * TT + rtid);
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    __syncwarp();  // the warp is done with the copy this one replaces (two tiles back)
+                    reinterpret_cast<float4 *>(s_lse[rs.idx][quarter])[lane] = lse_mine;
+                    if (j < j1) lse_mine = __ldg(reinterpret_cast<const float4 *>(lse_row + (j + 1) * TT) + lane);
+                    __syncwarp();
                 }
                 bar_wait(s_full + rs.idx, rs.phase, dead, &s_abort);
                 fence_after();
@@ -456,7 +458,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                 if (lane == 0) bar_arrive(s_empty + rs.idx);
                                 released = true;
                             }
-                            col_sum += colsum_block<64>(v, &s_lse[rs.idx][half * 64], sc, false, lane);
+                            col_sum += colsum_block<64>(v, &s_lse[rs.idx][quarter][half * 64], sc, false, lane);
                         }
                     }
                 } else {
@@ -472,7 +474,7 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             }
                             lse_block<32>(v, sc, fast, run_max, run_sum);
                         } else {
-                            col_sum += colsum_block<32>(v, &s_lse[rs.idx][cblk * 32], sc, edge, lane);
+                            col_sum += colsum_block<32>(v, &s_lse[rs.idx][quarter][cblk * 32], sc, edge, lane);
                         }
                     }
                 }
