@@ -158,6 +158,7 @@ __global__ void head_mean_kernel(const float *__restrict__ partial, int H, int N
                                  float *__restrict__ scores)
 {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    dependent_entry();  // launched as a programmatic dependent of the pass that writes `partial`
     if (i >= total) return;
     size_t seg = i / N;
     int n = (int)(i % N);
@@ -168,8 +169,13 @@ __global__ void head_mean_kernel(const float *__restrict__ partial, int H, int N
 
 int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, cudaStream_t st)
 {
-    head_mean_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(partial, H, N, total, scores);
-    return check_launch("head_mean_kernel");
+    cudaError_t e = launch_dependent(head_mean_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
+                                     partial, H, N, total, scores);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "head_mean_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
 
 template <typename T, int D>

@@ -313,6 +313,9 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     __syncthreads();
     fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched as a programmatic dependent: everything above (barriers, tensor memory) was set up
+    // while the kernel before it drained; its results (Q, K, the normalisers) are read from here on.
+    dependent_entry();
 
     if (warp == 0) {
         // ---- TMA producer ---------------------------------------------------------------------
@@ -569,8 +572,12 @@ int launch_pass(const CUtensorMap &mq, const CUtensorMap &mk, const ScoreArgs &a
     // fixed stride, 296 CTAs and 16 tiles per head left every CTA two tile indices only, and the
     // slowest did 12 tiles per item against a mean of 8.5).
     const int grid = items < 2 * sms ? items : 2 * sms;
-    score_tile_kernel<PASS, D><<<grid, 192, smem, st>>>(mq, mk, a);
-    return check_launch(PASS == 1 ? "score_tile_kernel<1>" : "score_tile_kernel<2>");
+    cudaError_t e = launch_dependent(score_tile_kernel<PASS, D>, dim3(grid), dim3(192), smem, st, mq, mk, a);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, PASS == 1 ? "score_tile_kernel<1>" : "score_tile_kernel<2>");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
 
 }  // namespace
