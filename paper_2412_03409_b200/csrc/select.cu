@@ -63,6 +63,32 @@ sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t 
     }
     __syncthreads();
 
+    if (P == nthr) {
+        // One key per thread, in a register: partners less than a warp apart exchange by shuffle,
+        // the others through shared memory, two buffers in turn so that one barrier per such step
+        // is enough.  (15 barriers instead of 55 for 1024 keys.)
+        uint64_t key = keys[tid];
+        uint64_t *buf[2] = {keys, keys + P};
+        int cur = 1;  // keys[] itself was read above, before the barrier
+        for (int k = 2; k <= P; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                uint64_t other;
+                if (j >= 32) {
+                    buf[cur][tid] = key;
+                    __syncthreads();
+                    other = buf[cur][tid ^ j];
+                    cur ^= 1;
+                } else {
+                    other = __shfl_xor_sync(0xffffffffu, key, j);
+                }
+                const bool keep_min = ((tid & j) == 0) == ((tid & k) == 0);
+                key = keep_min ? (key < other ? key : other) : (key > other ? key : other);
+            }
+        }
+        __syncthreads();  // every read of keys[] / the buffers is over
+        keys[tid] = key;
+        __syncthreads();
+    } else
     for (int k = 2; k <= P; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             for (int i = tid; i < (P >> 1); i += nthr) {
@@ -289,7 +315,7 @@ static int launch_sort(const pkv_shape *s, const float *scores, int32_t *order, 
     int P = 32;
     while (P < N) P <<= 1;
     int nthr = P < 1024 ? P : 1024;
-    size_t smem = (size_t)P * sizeof(uint64_t);
+    size_t smem = (size_t)P * sizeof(uint64_t) * (P == nthr ? 2 : 1);  // one key per thread: two exchange buffers
     static bool attr_done[64] = {};
     if (smem > 48 * 1024) {
         int rc = ensure_dynamic_smem((const void *)sort_scan_kernel, 128 * 1024, attr_done);
