@@ -385,7 +385,13 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         const int g = lane / LPR, c = lane % LPR;
         const int h0 = warp * HPW;  // H is a multiple of HPW (checked by the launcher)
         const uint32_t lane_off = (uint32_t)h0 * D * sizeof(T) + c * 16;
-        float qf[HPW][EPL], acc[HPW][EPL], m[HPW], l[HPW];
+        // Four heads per warp: q stays in its shared-memory buffer for the piece and a head's slice is
+        // re-read for every unit, which keeps that variant inside its 96 registers.
+        constexpr bool kQSmem = HPW >= 4;
+        float qf[kQSmem ? 1 : HPW][kQSmem ? 1 : EPL], acc[HPW][EPL], m[HPW], l[HPW];
+        const unsigned char *q_held = nullptr;
+        int q_held_idx = 0;
+        float q_scale = 0.f;
         Ring r{0, a.nstages, 0u};
         int qi = 0;
         uint32_t qph = 0;
@@ -422,13 +428,19 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                         Vec<T>::unpack(*reinterpret_cast<const uint4 *>(qb + (size_t)h * D * sizeof(T) + (v * LPR + c) * 16), x);
 #pragma unroll
                         for (int i = 0; i < VE; ++i) {
-                            qf[hh][v * VE + i] = x[i] * sc;
+                            if constexpr (!kQSmem) qf[hh][v * VE + i] = x[i] * sc;
                             acc[hh][v * VE + i] = 0.f;
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(qempty + qi);
+                if constexpr (kQSmem) {
+                    q_held = qb + (size_t)h0 * D * sizeof(T) + c * 16;
+                    q_held_idx = qi;
+                    q_scale = sc;
+                } else {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(qempty + qi);
+                }
                 qi ^= 1;
                 if (qi == 0) qph ^= 1u;
             }
@@ -445,9 +457,22 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                 const unsigned char *kb = ring + (uint32_t)r.slot * slot_bytes;
                 const unsigned char *kl = kb + (uint32_t)g * rb + lane_off;
 #pragma unroll
-                for (int j = 0; j < RPG; ++j) {
+                for (int hh = 0; hh < HPW; ++hh) {
+                    float qv[EPL];  // this head's slice of the scaled query
 #pragma unroll
-                    for (int hh = 0; hh < HPW; ++hh) {
+                    for (int v = 0; v < NV; ++v) {
+                        if constexpr (kQSmem) {
+                            float x[VE];
+                            Vec<T>::unpack(*reinterpret_cast<const uint4 *>(q_held + hh * (int)(D * sizeof(T)) + v * LPR * 16), x);
+#pragma unroll
+                            for (int i = 0; i < VE; ++i) qv[v * VE + i] = x[i] * q_scale;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < VE; ++i) qv[v * VE + i] = qf[hh][v * VE + i];
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j) {
                         float d0 = 0.f, d1 = 0.f;
                         if (whole || g + j * GPW < cnt) {
                             const unsigned char *row = kl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
@@ -457,8 +482,8 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                                 Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
 #pragma unroll
                                 for (int i = 0; i < VE; i += 2) {
-                                    d0 = fmaf(qf[hh][v * VE + i], x[i], d0);
-                                    d1 = fmaf(qf[hh][v * VE + i + 1], x[i + 1], d1);
+                                    d0 = fmaf(qv[v * VE + i], x[i], d0);
+                                    d1 = fmaf(qv[v * VE + i + 1], x[i + 1], d1);
                                 }
                             }
                         }
@@ -541,6 +566,10 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
 
             if (seg_end || u == u1 - 1) {
                 // ---- close this CTA's piece of the segment ---------------------------------------
+                if constexpr (kQSmem) {  // q was read in place until here
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(qempty + q_held_idx);
+                }
                 const int c_first = unit_owner(P[si], upc, rem), c_last = unit_owner(P[si + 1] - 1, upc, rem);
                 const int ncontrib = c_last - c_first + 1;
 #pragma unroll
@@ -909,7 +938,7 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     const size_t es = esize(s);
     const uint32_t row_bytes = (uint32_t)((size_t)H * D * es);
     int ur = 0, nstages = 0;
-    for (int cand = 8; cand >= 4 && !ur; cand >>= 1) {
+    for (int cand = 8; cand >= 2 && !ur; cand >>= 1) {  // rows per unit: as many as leave three ring stages
         int ns = kMaxStages;
         while (ns >= 3 && stream_smem_bytes(ns, cand, row_bytes, nact) > (size_t)kDynSmemMax) --ns;
         if (ns >= 3) {
@@ -979,7 +1008,10 @@ int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const 
     PKV_V(T, DD, 16, 4, 8, 544); \
     PKV_V(T, DD, 16, 2, 4, 544); \
     PKV_V(T, DD, 16, 4, 4, 384); \
-    PKV_V(T, DD, 16, 4, 4, 544)
+    PKV_V(T, DD, 16, 4, 4, 544); \
+    PKV_V(T, DD, 16, 2, 2, 544); \
+    PKV_V(T, DD, 16, 4, 2, 384); \
+    PKV_V(T, DD, 16, 4, 2, 544)
     if (bf && D == 128) {
         PKV_NARROW1(__nv_bfloat16, 128);
         PKV_WIDE(__nv_bfloat16, 128);
