@@ -456,38 +456,57 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
                 wait_phase(full + r.slot, r.phase, dead, &s_abort);
                 const unsigned char *kb = ring + (uint32_t)r.slot * slot_bytes;
                 const unsigned char *kl = kb + (uint32_t)g * rb + lane_off;
+                if constexpr (kQSmem) {
 #pragma unroll
-                for (int hh = 0; hh < HPW; ++hh) {
-                    float qv[EPL];  // this head's slice of the scaled query
+                    for (int hh = 0; hh < HPW; ++hh) {
+                        float qv[EPL];  // this head's slice of the scaled query
 #pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        if constexpr (kQSmem) {
+                        for (int v = 0; v < NV; ++v) {
                             float x[VE];
                             Vec<T>::unpack(*reinterpret_cast<const uint4 *>(q_held + hh * (int)(D * sizeof(T)) + v * LPR * 16), x);
 #pragma unroll
                             for (int i = 0; i < VE; ++i) qv[v * VE + i] = x[i] * q_scale;
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < VE; ++i) qv[v * VE + i] = qf[hh][v * VE + i];
                         }
-                    }
 #pragma unroll
-                    for (int j = 0; j < RPG; ++j) {
-                        float d0 = 0.f, d1 = 0.f;
-                        if (whole || g + j * GPW < cnt) {
-                            const unsigned char *row = kl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
+                        for (int j = 0; j < RPG; ++j) {
+                            float d0 = 0.f, d1 = 0.f;
+                            if (whole || g + j * GPW < cnt) {
+                                const unsigned char *row = kl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
 #pragma unroll
-                            for (int v = 0; v < NV; ++v) {
-                                float x[VE];
-                                Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
+                                for (int v = 0; v < NV; ++v) {
+                                    float x[VE];
+                                    Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
 #pragma unroll
-                                for (int i = 0; i < VE; i += 2) {
-                                    d0 = fmaf(qv[v * VE + i], x[i], d0);
-                                    d1 = fmaf(qv[v * VE + i + 1], x[i + 1], d1);
+                                    for (int i = 0; i < VE; i += 2) {
+                                        d0 = fmaf(qv[v * VE + i], x[i], d0);
+                                        d1 = fmaf(qv[v * VE + i + 1], x[i + 1], d1);
+                                    }
                                 }
                             }
+                            s[hh][j] = d0 + d1;
                         }
-                        s[hh][j] = d0 + d1;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < RPG; ++j) {
+#pragma unroll
+                        for (int hh = 0; hh < HPW; ++hh) {
+                            float d0 = 0.f, d1 = 0.f;
+                            if (whole || g + j * GPW < cnt) {
+                                const unsigned char *row = kl + (uint32_t)(j * GPW) * rb + hh * (int)(D * sizeof(T));
+#pragma unroll
+                                for (int v = 0; v < NV; ++v) {
+                                    float x[VE];
+                                    Vec<T>::unpack(*reinterpret_cast<const uint4 *>(row + v * LPR * 16), x);
+#pragma unroll
+                                    for (int i = 0; i < VE; i += 2) {
+                                        d0 = fmaf(qf[hh][v * VE + i], x[i], d0);
+                                        d1 = fmaf(qf[hh][v * VE + i + 1], x[i + 1], d1);
+                                    }
+                                }
+                            }
+                            s[hh][j] = d0 + d1;
+                        }
                     }
                 }
 #pragma unroll
