@@ -56,7 +56,7 @@ def measured_peaks():
 # DRAM bytes (read + write) of one decode_stream_kernel launch from an ncu capture (its summary is
 # kept under profiles/), keyed by workload, with the hash of the kernel's source
 # the counters were taken on: once that file changes the figure is stale and `traffic` reads null.
-DECODE_TRAFFIC = {"llava7b_b1": (102.61e6, "466a79f38ed17f1d")}
+DECODE_TRAFFIC = {"llava7b_b1": (102.61e6, "074b548178a7e41a")}
 
 
 def decode_traffic(workload):

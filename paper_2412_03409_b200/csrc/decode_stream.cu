@@ -385,9 +385,10 @@ __global__ void __launch_bounds__(MAXT, 1) decode_stream_kernel(const DecodeArgs
         const int g = lane / LPR, c = lane % LPR;
         const int h0 = warp * HPW;  // H is a multiple of HPW (checked by the launcher)
         const uint32_t lane_off = (uint32_t)h0 * D * sizeof(T) + c * 16;
-        // Four heads per warp: q stays in its shared-memory buffer for the piece and a head's slice is
-        // re-read for every unit, which keeps that variant inside its 96 registers.
-        constexpr bool kQSmem = HPW >= 4;
+        // Four heads per warp in a block of more than 12 warps (96 registers per thread): q stays in its
+        // shared-memory buffer for the piece and a head's slice is re-read for every unit, which keeps
+        // that variant free of spills.  With fewer warps there is room for q in registers.
+        constexpr bool kQSmem = HPW >= 4 && MAXT > 384;
         float qf[kQSmem ? 1 : HPW][kQSmem ? 1 : EPL], acc[HPW][EPL], m[HPW], l[HPW];
         const unsigned char *q_held = nullptr;
         int q_held_idx = 0;
