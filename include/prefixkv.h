@@ -94,9 +94,12 @@ const char *prefixkv_last_cuda_error(void);
  *               causal logits, if the caller's prefill attention kept it; when
  *               NULL the library computes it in a first pass
  *   scores      [B,L,N] fp32, out
- * bf16 inputs use tensor cores with fp32 accumulation; fp32 inputs use fp32 FMA.
+ * bf16 inputs use tensor cores with fp32 accumulation; fp32 inputs use fp32 FMA (so do
+ * bf16 inputs whose strides no tensor map can describe, e.g. a zero stride).
  * The workspace holds per-head partial sums and work counters: calls that share one must
- * not overlap on the GPU.
+ * not overlap on the GPU.  The call has no status argument: if a bounded wait inside the
+ * tensor-core kernel runs out, every score of the call is written as NaN, which
+ * prefixkv_search / prefixkv_apply_lengths report as PKV_DEV_BAD_SCORE.
  */
 int prefixkv_score(const pkv_shape *shape, const void *q, pkv_strides qs, const void *k,
                    pkv_strides ks, const float *layer_scale, const float *lse, float *scores,
@@ -269,6 +272,17 @@ int prefixkv_decode_attn_static(const pkv_shape *shape, pkv_cache *cache, const 
  *   cum  [B,L,N] from prefixkv_search;  gini [B,L] fp64 out
  */
 int prefixkv_gini(const pkv_shape *shape, const uint64_t *cum, double *gini, void *cuda_stream);
+
+/*
+ * Self-test of the bounded waits (a robustness aid; the paper has no counterpart).  Every
+ * wait on an mbarrier inside the tensor-core scoring kernel (which = 0) and the streaming
+ * decode kernel (which = 1) gives up after a fixed number of tries; the kernel then stops
+ * waiting, finishes in bounds and reports.  This call runs that give-up path alone: one warp
+ * waits, with a limit of a few thousand tries (milliseconds), on a barrier that nothing
+ * completes, and dev_status[0] is raised to PKV_DEV_TIMEOUT.  Nothing faults or hangs.
+ *   dev_status  [>= 1] int32, must hold PKV_DEV_OK on entry for the code to be recorded
+ */
+int prefixkv_selftest_bounded_wait(int32_t which, int32_t *dev_status, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -69,6 +69,17 @@ def score_layer(q, k, scale, want_f64=False):
     return (out, out64) if want_f64 else out
 
 
+def lse_layer(q, k, scale):
+    """Natural-log normaliser of every query's causal softmax.  q, k: [H, N, D] -> [H, N] fp64."""
+    q, k = _f32(q), _f32(k)
+    H, N, D = q.shape
+    assert k.shape == q.shape
+    out = np.empty((H, N), np.float64)
+    _L().orc_lse_layer(_p(q, ctypes.c_float), _p(k, ctypes.c_float), H, N, D,
+                       ctypes.c_double(float(scale)), _p(out, ctypes.c_double))
+    return out
+
+
 def sort_desc(scores):
     """Priority sequence s_l^1..s_l^N: positions by (importance desc, position asc)."""
     scores = _f32(scores)

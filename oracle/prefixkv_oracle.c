@@ -15,7 +15,8 @@
  * information-retention ratio, R_l retained ratio (here the integer R_l * N).
  *
  * Pins (tests/test_oracle_*.py): harmonic-number closed form and softmax
- * column sums via a library softmax for the score; library stable sort for the
+ * column sums via a library softmax for the score; a library log-sum-exp and
+ * the closed form log(m) for zero queries for the normaliser; library stable sort for the
  * order; exact rational arithmetic for the cumulative weights; brute-force
  * enumeration of every breakpoint of p and a hand-worked example for the
  * search; library dense attention for decode.  Unpinned: nothing in this file
@@ -73,6 +74,37 @@ void orc_score_layer(const float *q, const float *k, int H, int N, int D,
     }
     free(s);
     free(col);
+}
+
+/* ------------------------------------------------------------------------
+ * Normaliser of the same softmax, Sec. 3.2: for every head i and query m the
+ * natural logarithm of sum over keys j <= m of exp(scale * (q^{i,m} . k^{i,j})),
+ * i.e. the denominator of a_l^{i,m,n} in the log domain.  A prefill attention
+ * kernel usually keeps exactly this value per query; the library accepts it in
+ * place of recomputing it.  q, k: [H][N][D]; out: [H][N] fp64.
+ * ---------------------------------------------------------------------- */
+void orc_lse_layer(const float *q, const float *k, int H, int N, int D, double scale,
+                   double *out)
+{
+    double *s = (double *)malloc((size_t)N * sizeof(double));
+    for (int i = 0; i < H; ++i) {
+        const float *qh = q + (size_t)i * N * D;
+        const float *kh = k + (size_t)i * N * D;
+        for (int m = 0; m < N; ++m) {
+            double mx = -INFINITY;
+            for (int j = 0; j <= m; ++j) {
+                double dot = 0.0;
+                for (int d = 0; d < D; ++d)
+                    dot += (double)qh[(size_t)m * D + d] * (double)kh[(size_t)j * D + d];
+                s[j] = scale * dot;
+                if (s[j] > mx) mx = s[j];
+            }
+            double z = 0.0;
+            for (int j = 0; j <= m; ++j) z += exp(s[j] - mx);
+            out[(size_t)i * N + m] = mx + log(z);
+        }
+    }
+    free(s);
 }
 
 /* ------------------------------------------------------------------------

@@ -25,7 +25,7 @@ EXPORTS = ["prefixkv_workspace_bytes", "prefixkv_last_cuda_error", "prefixkv_sco
            "prefixkv_search", "prefixkv_apply_lengths", "prefixkv_compact",
            "prefixkv_decode_attn", "prefixkv_gini", "prefixkv_rescale",
            "prefixkv_estimate_config", "prefixkv_decode_attn_static",
-           "prefixkv_decode_static_limit_bytes"]
+           "prefixkv_selftest_bounded_wait", "prefixkv_decode_static_limit_bytes"]
 
 
 class Shape(ctypes.Structure):
@@ -76,6 +76,7 @@ def _load():
     lib.prefixkv_estimate_config.argtypes = [sp, vp, i64, vp, vp, vp]
     lib.prefixkv_decode_attn_static.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp,
                                                 i32, i32, vp, vp, vp]
+    lib.prefixkv_selftest_bounded_wait.argtypes = [i32, vp, vp]
     for name in EXPORTS[2:-1]:
         getattr(lib, name).restype = ctypes.c_int
     lib.prefixkv_decode_static_limit_bytes.restype = ctypes.c_size_t
@@ -246,3 +247,8 @@ def prefixkv_estimate_config(shape, length, budget_rows, len_out, dev_status):
     _check(_lib.prefixkv_estimate_config(ctypes.byref(shape), _ptr(length), int(budget_rows),
                                          _ptr(len_out), _ptr(dev_status), _stream()),
            "prefixkv_estimate_config")
+
+
+def prefixkv_selftest_bounded_wait(which, dev_status):
+    _check(_lib.prefixkv_selftest_bounded_wait(int(which), _ptr(dev_status), _stream()),
+           "prefixkv_selftest_bounded_wait")

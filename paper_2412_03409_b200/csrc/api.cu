@@ -57,6 +57,8 @@ int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const voi
 bool score_tc_usable(const pkv_shape *s, const void *q, pkv_strides qs, const void *k, pkv_strides ks);
 
 size_t score_tc_ws_bytes(const pkv_shape *s);
+int selftest_wait_score(int32_t *dev_status, cudaStream_t st);
+int selftest_wait_stream(int32_t *dev_status, cudaStream_t st);
 
 static size_t score_ws_bytes(const pkv_shape *s)
 {
@@ -150,4 +152,12 @@ extern "C" int prefixkv_gini(const pkv_shape *shape, const uint64_t *cum, double
     gini_kernel<<<shape->batch * shape->layers, 256, 0, (cudaStream_t)cuda_stream>>>(
         cum, shape->prompt_len, gini);
     return check_launch("gini_kernel");
+}
+
+extern "C" int prefixkv_selftest_bounded_wait(int32_t which, int32_t *dev_status, void *cuda_stream)
+{
+    if (!dev_status) return PKV_ERR_INVALID_ARG;
+    if (which == 0) return selftest_wait_score(dev_status, (cudaStream_t)cuda_stream);
+    if (which == 1) return selftest_wait_stream(dev_status, (cudaStream_t)cuda_stream);
+    return PKV_ERR_INVALID_ARG;
 }

@@ -60,7 +60,7 @@ decode_partial_kernel(const T *__restrict__ q, const T *__restrict__ k_new, cons
     const int b = blockIdx.y / nl, l = layer_begin + blockIdx.y % nl;
     const int seg = b * L + l;
     const int n = len[seg];
-    if (n + 1 > cap[seg]) {
+    if (n < 1 || n + 1 > cap[seg]) {  // never compacted, or full: reported, zero output, length kept
         if (threadIdx.x == 0 && sp == 0) raise_status(dev_status, b, PKV_DEV_CAPACITY);
         return;
     }
@@ -126,7 +126,7 @@ decode_merge_kernel(const float *__restrict__ part_acc, const float *__restrict_
     const int b = blockIdx.x / nl, l = layer_begin + blockIdx.x % nl;
     const int seg = b * L + l;
     const int n = len[seg];
-    const bool full = n + 1 > cap[seg];
+    const bool full = n < 1 || n + 1 > cap[seg];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int h = warp; h < H; h += 8) {
         float o[EPL];

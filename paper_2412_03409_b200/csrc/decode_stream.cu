@@ -78,9 +78,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait: false when the limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t limit = kSpinLimit)
 {
-    for (uint32_t i = 0; i < kSpinLimit; ++i)
+    for (uint32_t i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -139,13 +139,39 @@ __device__ __forceinline__ int unit_owner(int u, int q, int rem)
 
 // Wait for a barrier phase; `dead` latches once a bounded wait has run out anywhere in
 // the CTA, after which nothing waits any more (the results are then unspecified).
-__device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag)
+__device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag,
+                                           uint32_t limit = kSpinLimit)
 {
     if (dead || mbar_try_wait(bar, parity)) return;
-    if (*(volatile int *)abort_flag || !mbar_wait(bar, parity)) {
+    if (*(volatile int *)abort_flag || !mbar_wait(bar, parity, limit)) {
         dead = true;
         atomicExch(abort_flag, 1);
     }
+}
+
+// One warp waits, with a short limit, on a barrier phase that nothing completes: the give-up path
+// of the streaming kernel in isolation.
+__global__ void selftest_wait_stream_kernel(int32_t *dev_status, uint32_t limit)
+{
+    __shared__ uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool dead = false;
+    if (threadIdx.x == 0) wait_phase(&bar, 0u, dead, &s_abort, limit);
+    __syncthreads();
+    wait_phase(&bar, 0u, dead, &s_abort, limit);  // the other lanes see the flag and stop at once
+    if (threadIdx.x == 0 && dead && s_abort) raise_status(dev_status, 0, PKV_DEV_TIMEOUT);
+}
+
+int selftest_wait_stream(int32_t *dev_status, cudaStream_t st)
+{
+    selftest_wait_stream_kernel<<<1, 32, 0, st>>>(dev_status, 4096u);
+    return check_launch("selftest_wait_stream_kernel");
 }
 
 // What this step does to active segment si: the rows it attends over (the new row included),

@@ -154,12 +154,18 @@ score_colsum_kernel(const T *__restrict__ q, pkv_strides qs, const T *__restrict
 }
 
 // scores[seg, n] = (1/H) * sum_h partial[seg, h, n], heads in index order.
+// A set abort word (a bounded wait of the tensor-core passes ran out, so `partial` is not to be
+// trusted) turns every score into NaN, which the selection stage reports as PKV_DEV_BAD_SCORE.
 __global__ void head_mean_kernel(const float *__restrict__ partial, int H, int N, size_t total,
-                                 float *__restrict__ scores)
+                                 float *__restrict__ scores, const int32_t *__restrict__ abort_word)
 {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     dependent_entry();  // launched as a programmatic dependent of the pass that writes `partial`
     if (i >= total) return;
+    if (abort_word && *abort_word != 0) {
+        scores[i] = __int_as_float(0x7fc00000);
+        return;
+    }
     size_t seg = i / N;
     int n = (int)(i % N);
     float t = 0.f;
@@ -167,10 +173,11 @@ __global__ void head_mean_kernel(const float *__restrict__ partial, int H, int N
     scores[i] = t / (float)H;
 }
 
-int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, cudaStream_t st)
+int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, const int32_t *abort_word,
+                     cudaStream_t st)
 {
     cudaError_t e = launch_dependent(head_mean_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                                     partial, H, N, total, scores);
+                                     partial, H, N, total, scores, abort_word);
     if (e != cudaSuccess) {
         set_cuda_error(e, "head_mean_kernel");
         return PKV_ERR_CUDA;
@@ -202,7 +209,7 @@ int launch_score_simt(const pkv_shape *s, const void *q, pkv_strides qs, const v
                                                     N, lse, lse_mul, partial);
     int rc = check_launch("score_colsum_kernel");
     if (rc != PKV_OK) return rc;
-    return launch_head_mean(partial, H, N, (size_t)B * L * N, scores, st);
+    return launch_head_mean(partial, H, N, (size_t)B * L * N, scores, nullptr, st);
 }
 
 #define PKV_INST(T, D)                                                                            \

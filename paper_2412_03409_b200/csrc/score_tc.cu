@@ -18,7 +18,8 @@
 // tile and the tiles streamed against it) come from a device counter: the TMA thread takes the
 // next number and announces it to the other roles through a four-entry shared-memory queue,
 // so CTAs that run faster do more.  Every mbarrier wait is bounded: when one runs out the CTA
-// stops waiting, reports PKV_DEV_TIMEOUT and still releases its tensor memory.
+// stops waiting, sets the call's abort word (the head mean then writes NaN for every score, which
+// the selection stage reports as PKV_DEV_BAD_SCORE) and still releases its tensor memory.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -37,8 +38,8 @@ struct ScoreArgs {
     const float *layer_scale;
     float *lse2;     // [B*L*H][Npad] log2-sum-exp of scaled logits, +inf beyond N
     float *partial;  // [B*L*H][N] per-head column sums
-    int32_t *abort_word;  // device word set when a bounded wait runs out (may be null)
-    int *next_item;       // [2] work counters, one per pass; zeroed before the first pass is launched
+    int32_t *abort_word;  // device word set when a bounded wait runs out: the head mean then writes NaN scores
+    int *next_item;       // [2] work counters, one per pass; zeroed, with the abort word, before the first pass
     int L, H, N, Npad, tiles, nseg;
 };
 
@@ -70,10 +71,11 @@ __device__ __forceinline__ bool bar_try(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  `dead` latches for the calling thread once any wait in the CTA has run out.
-__device__ __forceinline__ void bar_wait(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag)
+__device__ __forceinline__ void bar_wait(uint64_t *bar, uint32_t parity, bool &dead, int *abort_flag,
+                                         uint32_t limit = kSpin)
 {
     if (dead) return;
-    for (uint32_t i = 0; i < kSpin; ++i) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (bar_try(bar, parity)) return;
         if ((i & 255u) == 255u && *(volatile int *)abort_flag) break;
     }
@@ -494,16 +496,37 @@ score_tile_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 a.partial[(size_t)sh * a.N + grow] = col_sum;
             }
         }
-        if (dead && lane == 0 && a.abort_word) atomicExch(a.abort_word, (int)PKV_DEV_TIMEOUT);
     }
+    // Any role whose wait ran out has set s_abort; one thread passes it on (after the barrier below).
 
     fence_before();
     __syncthreads();
     fence_after();
+    if (tid == 0 && s_abort && a.abort_word) atomicExch(a.abort_word, (int)PKV_DEV_TIMEOUT);
     if (warp == 1) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
     }
+}
+
+// One warp waits, with a short limit, on a barrier phase that nothing completes: the wait gives
+// up, latches `dead`, and the status word reads PKV_DEV_TIMEOUT.  This is the whole give-up path
+// of the kernel above in isolation (its roles then stop waiting, drain and release tensor memory).
+__global__ void selftest_wait_kernel(int32_t *dev_status, uint32_t limit)
+{
+    __shared__ uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        bar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool dead = false;
+    if (threadIdx.x == 0) bar_wait(&bar, 0u, dead, &s_abort, limit);
+    __syncthreads();
+    bar_wait(&bar, 0u, dead, &s_abort, limit);  // the other lanes see the flag and stop at once
+    if (threadIdx.x == 0 && dead && s_abort) raise_status(dev_status, 0, PKV_DEV_TIMEOUT);
 }
 
 // Caller-supplied natural-log lse [B*L*H][N] -> padded log2 layout.
@@ -582,7 +605,14 @@ int launch_pass(const CUtensorMap &mq, const CUtensorMap &mk, const ScoreArgs &a
 
 }  // namespace
 
-int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, cudaStream_t st);
+int launch_head_mean(const float *partial, int H, int N, size_t total, float *scores, const int32_t *abort_word,
+                     cudaStream_t st);
+
+int selftest_wait_score(int32_t *dev_status, cudaStream_t st)
+{
+    selftest_wait_kernel<<<1, 32, 0, st>>>(dev_status, 2000u);  // each try may sleep up to kSuspendNs
+    return check_launch("selftest_wait_kernel");
+}
 
 bool score_tc_usable(const pkv_shape *s, const void *, pkv_strides, const void *, pkv_strides)
 {
@@ -594,7 +624,7 @@ size_t score_tc_ws_bytes(const pkv_shape *s)
     const size_t rows = (size_t)s->batch * s->layers * s->heads;
     const size_t npad = ((size_t)s->prompt_len + TT - 1) / TT * TT;
     return round_up(rows * s->prompt_len * sizeof(float), kWsAlign) + round_up(rows * npad * sizeof(float), kWsAlign) +
-           kWsAlign;  // the two work counters
+           kWsAlign;  // the two work counters and the abort word
 }
 
 // Returns PKV_OK, an error, or -1 when the tensor maps cannot describe the caller's layout.
@@ -609,13 +639,13 @@ int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const voi
     a.layer_scale = scale;
     a.partial = (float *)ws;
     a.lse2 = (float *)((unsigned char *)ws + round_up(rows * N * sizeof(float), kWsAlign));
-    a.abort_word = nullptr;
     a.L = L; a.H = H; a.N = N;
     a.tiles = (N + TT - 1) / TT;
     a.Npad = a.tiles * TT;
     a.next_item = (int *)((unsigned char *)a.lse2 + round_up(rows * a.Npad * sizeof(float), kWsAlign));
+    a.abort_word = a.next_item + 2;
     {
-        cudaError_t e = cudaMemsetAsync(a.next_item, 0, 2 * sizeof(int), st);
+        cudaError_t e = cudaMemsetAsync(a.next_item, 0, 4 * sizeof(int), st);
         if (e != cudaSuccess) {
             set_cuda_error(e, "cudaMemsetAsync(score work counters)");
             return PKV_ERR_CUDA;
@@ -646,7 +676,7 @@ int launch_score_tc(const pkv_shape *s, const void *q, pkv_strides qs, const voi
     if (rc != PKV_OK) return rc;
     rc = s->head_dim == 128 ? launch_pass<2, 128>(mq, mk, a, sms, st) : launch_pass<2, 64>(mq, mk, a, sms, st);
     if (rc != PKV_OK) return rc;
-    return launch_head_mean(a.partial, H, N, (size_t)B * L * N, scores, st);
+    return launch_head_mean(a.partial, H, N, (size_t)B * L * N, scores, a.abort_word, st);
 }
 
 }  // namespace pkv

@@ -309,10 +309,11 @@ def test_decode_with_stale_workspace(api, byte):
     assert a.status.cpu().tolist() == b.status.cpu().tolist() == [0]
 
 
-def test_decode_empty_segment_is_reported(api):
+@pytest.mark.parametrize("kw", [dict(H=4), dict(H=72, D=64)])      # streaming kernel; two-kernel path (H > 64)
+def test_decode_empty_segment_is_reported(api, kw):
     """A segment with no rows (never compacted) cannot be attended over: the sample's status says
     so, its output is zero, its length stays, and the other segments are unaffected."""
-    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], B=2, L=3, H=4, N=80, T=2)
+    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], B=2, L=3, N=80, T=2, **kw)
     q, k, v = wl.make_prompt(w, "cuda")
     scale = wl.layer_scale(w)
     scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 11) for b in range(w.B)])
@@ -425,18 +426,40 @@ def test_score_token_major_layout(api, name, kw):
         check_scores(got[b, l].cpu().numpy(), r, SCORE_TOL[w.dtype])
 
 
-def test_score_with_caller_lse(api):
-    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=2, H=4, N=160)
+@pytest.mark.parametrize("name,kw", [
+    ("llava7b_b1", dict(L=2, H=4, N=300)),           # bf16: tensor-core pass 2 on a converted lse
+    ("llava7b_b16", dict(B=2, L=1, H=3, N=129, D=64)),
+    ("tiny", dict(N=150, H=3, L=2)),                 # fp32: FMA pass 2 with the natural-log lse
+    ("tiny", dict(N=70, H=2, L=1, D=128)),
+])
+def test_score_with_caller_lse(api, name, kw):
+    """The log-sum-exp a prefill kernel would have kept is taken from the oracle (fp64, rounded
+    once to fp32); the scores computed from it must meet the same bar against the oracle."""
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
     q, k, v = wl.make_prompt(w, "cuda")
     scale = wl.layer_scale(w)
     s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
-    base = s.score(q, k).clone()
-    logits = torch.einsum("blhmd,blhnd->blhmn", q.float(), k.float()) * \
-        torch.from_numpy(scale).cuda().view(1, -1, 1, 1, 1)
-    mask = torch.ones(w.N, w.N, dtype=torch.bool, device="cuda").tril()
-    lse = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1).contiguous()
-    got = s.score(q, k, lse=lse)
-    assert (got - base).abs().max() <= 2e-3 * base.abs().max()
+    lse = np.stack([np.stack([oracle.lse_layer(to_np32(q[b, l]), to_np32(k[b, l]), float(scale[l]))
+                              for l in range(w.L)]) for b in range(w.B)])
+    lse_dev = torch.from_numpy(lse.astype(np.float32)).cuda()
+    s.scores.fill_(float("nan"))
+    got = s.score(q, k, lse=lse_dev).cpu().numpy()
+    for (b, l), r in oracle_scores(q, k, scale).items():
+        check_scores(got[b, l], r, SCORE_TOL[w.dtype])
+
+
+def test_score_bf16_layout_without_tensor_map(api):
+    """A bf16 K that is one prompt shared by both samples (batch stride 0) cannot be described by
+    a tensor map, so the call takes the FMA kernels with strided loads: same bar."""
+    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], B=2, L=2, H=3, N=100)
+    q, k, v = wl.make_prompt(w, "cuda")
+    kb = k[:1].expand(2, -1, -1, -1, -1)
+    assert kb.stride(0) == 0
+    scale = wl.layer_scale(w)
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=1)
+    got = s.score(q, kb).cpu().numpy()
+    for (b, l), r in oracle_scores(q, kb, scale).items():
+        check_scores(got[b, l], r, SCORE_TOL[w.dtype])
 
 
 # --------------------------------------------------------------------------
@@ -482,8 +505,16 @@ def test_gini_matches_oracle(api):
 def test_argument_validation_fails_on_the_host(api):
     s = _session(1, 2, 4, 64, 32, torch.float32, np.ones(2), decode_cap=1)
     bad = api.make_shape(1, 2, 4, 48, 32, torch.float32)       # unsupported head_dim
-    assert api.lib().prefixkv_search(bad, 1, 1, 0.0, 1, 0, 1, 1, 1, 1, 1, 1, None, 0, None) == \
-        api.PKV_ERR_UNSUPPORTED
+    # (real buffers of the session, sized for the same B, L, N: a refusal that ever moved behind
+    # a launch would fail the assertions below, not touch made-up addresses)
+    s.len.fill_(-5)
+    s.status.fill_(0)
+    p = lambda t: t.data_ptr()
+    rc = api.lib().prefixkv_search(bad, p(s.scores), p(s.budget), 0.0, 1, 0, p(s.order), p(s.cum), p(s.len),
+                                   p(s.p), p(s.iters), p(s.status), None, 0, None)
+    torch.cuda.synchronize()
+    assert rc == api.PKV_ERR_UNSUPPORTED
+    assert bool((s.len == -5).all()) and int(s.status.abs().sum()) == 0
     long = api.make_shape(1, 2, 4, 64, 16385, torch.float32)
     assert api.prefixkv_workspace_bytes(long, api.WS_SCORE) == 0
     with pytest.raises(api.PrefixKVError):
@@ -581,3 +612,17 @@ def test_decode_time_pruning_matches_oracle(api, name, kw, d):
         np.testing.assert_array_equal(to_np32(s.cache.k[o:o + len(st["k"])]), np.stack(st["k"]))
         np.testing.assert_array_equal(to_np32(s.cache.v[o:o + len(st["v"])]), np.stack(st["v"]))
         assert int(s.cache.gen[b * w.L + l]) == w.T
+
+
+# --------------------------------------------------------------------------
+# bounded waits give up and report, without faulting or hanging anything
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("which", [0, 1])
+def test_bounded_wait_reports_timeout(api, which):
+    """A warp waits on a barrier that nothing completes, with a limit of a few thousand tries:
+    the wait returns, the status word reads PKV_DEV_TIMEOUT and the context stays usable."""
+    status = torch.zeros(2, dtype=torch.int32, device="cuda")
+    api.prefixkv_selftest_bounded_wait(which, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [api.DEV_TIMEOUT, 0]
+    assert int((torch.arange(8, device="cuda") + 1).sum()) == 36      # later work runs normally

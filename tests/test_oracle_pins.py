@@ -91,6 +91,27 @@ def test_score_invariants():
     np.testing.assert_allclose(Id, I, rtol=1e-13)
 
 
+def test_lse_matches_library_and_closed_form():
+    """The per-query normaliser: torch.logsumexp over the masked logits; log(m) when every
+    logit of query m (1-based) is zero; and exp(logit - lse) column-summed reproduces the score."""
+    H, N, D, scale = 3, 41, 8, 0.8
+    rng = np.random.default_rng(77)
+    q = rng.standard_normal((H, N, D)).astype(np.float32)
+    k = rng.standard_normal((H, N, D)).astype(np.float32)
+    lse = oracle.lse_layer(q, k, scale)
+    logits = scale * torch.from_numpy(q).double() @ torch.from_numpy(k).double().transpose(1, 2)
+    mask = torch.ones(N, N, dtype=torch.bool).tril()
+    ref = torch.logsumexp(logits.masked_fill(~mask, float("-inf")), dim=-1).numpy()
+    np.testing.assert_allclose(lse, ref, rtol=1e-13, atol=1e-13)
+    zero = oracle.lse_layer(np.zeros_like(q), k, 1.0)
+    np.testing.assert_allclose(zero, np.log(np.arange(1, N + 1))[None].repeat(H, 0), rtol=1e-14, atol=1e-15)
+    # operand order matters (q^m . k^j with j <= m, not the transpose)
+    assert np.abs(oracle.lse_layer(k, q, scale) - lse).max() > 1e-3
+    probs = torch.exp(logits - torch.from_numpy(lse)[..., None]).masked_fill(~mask, 0.0)
+    _, I = oracle.score_layer(q, k, scale, want_f64=True)
+    np.testing.assert_allclose(probs.sum(dim=1).mean(dim=0).numpy(), I, rtol=1e-12)
+
+
 def test_score_single_token():
     q = np.full((2, 1, 4), 3.0, np.float32)
     assert oracle.score_layer(q, q, 1.0)[0] == 1.0

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2412_03409_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -41,6 +42,8 @@ def test_static_scratch_decode_matches_workspace_decode(name, kw):
     assert api.prefixkv_workspace_bytes(api.make_shape(w.B, w.L, w.H, w.D, w.N, w.dtype),
                                         api.WS_DECODE) <= api.prefixkv_decode_static_limit_bytes()
     ref, sta = _pair(w)
+    f32 = lambda t: t.detach().float().cpu().numpy()
+    scale = wl.layer_scale(w)
     for t in range(2):                                   # two calls in a row share the array
         qd, kn, vn = wl.make_decode_inputs(w, t, "cuda")
         want = ref.decode(qd, kn, vn).float().clone()
@@ -51,6 +54,13 @@ def test_static_scratch_decode_matches_workspace_decode(name, kw):
         assert torch.isfinite(got).all()
         assert (got - want).abs().max().item() <= DECODE_TOL[w.dtype]
         assert torch.equal(sta.cache.len, ref.cache.len)
+        # and against the oracle, over the rows the cache now holds (the new one included)
+        for seg in (0, w.B * w.L - 1):
+            b, l = divmod(seg, w.L)
+            o, n = int(sta.cache.row_offset[seg]), int(sta.cache.len[seg])
+            want64 = oracle.decode_attn(f32(qd[b, l]), f32(sta.cache.k[o:o + n]), f32(sta.cache.v[o:o + n]),
+                                        float(scale[l]))
+            assert np.abs(f32(got[b, l]) - want64).max() <= DECODE_TOL[w.dtype]
     assert sta.status.cpu().tolist() == [0] * w.B
     # the appended rows landed in the cache exactly as with the workspace call
     for seg in range(w.B * w.L):
@@ -61,10 +71,26 @@ def test_static_scratch_decode_matches_workspace_decode(name, kw):
 
 
 def test_static_scratch_decode_refuses_large_shapes():
+    """A shape whose scratch need is above the built-in array is refused on the host, before any
+    launch.  Every pointer handed over is a real (small) device buffer and the cache describes
+    exactly those buffers, so that if the refusal ever moved behind a launch this test would fail
+    an assertion below instead of sending a kernel to made-up addresses."""
     from paper_2412_03409_b200 import api
     big = api.make_shape(16, 32, 32, 128, 640, torch.bfloat16)
     assert api.prefixkv_workspace_bytes(big, api.WS_DECODE) > api.prefixkv_decode_static_limit_bytes()
-    cache = api.CacheStruct(16, 16, 16, 16, 16, 10, 1, 0, None, None, None)
-    rc = api.lib().prefixkv_decode_attn_static(big, cache, 16, 16, 16, 16, 0, 32, 16, 16, None)
+    nseg = 16 * 32
+    cache = api.alloc_cache(big, total_rows=0, decode_cap=1, device="cuda", fill=0.0)
+    assert cache.k.shape[0] == nseg                          # one row of head-room per segment, nothing else
+    cache.cap.fill_(1)
+    cache.row_offset.copy_(torch.arange(nseg + 1, dtype=torch.int64, device="cuda"))
+    x = torch.zeros((16, 32, 32, 128), dtype=torch.bfloat16, device="cuda")
+    out = torch.full_like(x, 7.0)
+    scale = torch.ones(32, dtype=torch.float32, device="cuda")
+    status = torch.zeros(16, dtype=torch.int32, device="cuda")
+    p = lambda t: t.data_ptr()
+    rc = api.lib().prefixkv_decode_attn_static(big, cache.c, p(x), p(x), p(x), p(scale), 0, 32, p(out),
+                                               p(status), None)
+    torch.cuda.synchronize()
     assert rc == api.PKV_ERR_STATIC_LIMIT
     assert b"16 MiB" in api.lib().prefixkv_last_cuda_error()
+    assert int(cache.len.abs().sum()) == 0 and bool((out == 7.0).all()) and int(status.abs().sum()) == 0
