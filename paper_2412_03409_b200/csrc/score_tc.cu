@@ -178,6 +178,12 @@ __device__ __forceinline__ float ex2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ void fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 
@@ -204,10 +210,14 @@ __device__ __forceinline__ void lse_block(float (&v)[NC], float sc, bool fast, f
 #pragma unroll
         for (int i = 0; i < NC; ++i) v[i] = v[i] == -INFINITY ? -INFINITY : v[i] * sc;
     }
-    float c4[4] = {v[0], v[1], v[2], v[3]};
+    // (three-input maximum: half the comparisons; the loop takes four values at a time, the last two come at the end)
+    float c2[2] = {v[0], v[1]};
 #pragma unroll
-    for (int i = 4; i < NC; ++i) c4[i & 3] = fmaxf(c4[i & 3], v[i]);
-    const float cmax = fmaxf(fmaxf(c4[0], c4[1]), fmaxf(c4[2], c4[3]));
+    for (int i = 2; i + 2 < NC; i += 4) {
+        c2[0] = max3(c2[0], v[i], v[i + 1]);
+        c2[1] = max3(c2[1], v[i + 2], v[i + 3]);
+    }
+    const float cmax = max3(c2[0], c2[1], fmaxf(v[NC - 2], v[NC - 1]));
     const float nm = fmaxf(run_max, fast ? cmax * sc : cmax);  // finite: column 0 is never masked
     float p4[4] = {0.f, 0.f, 0.f, 0.f};
     if (fast) {
