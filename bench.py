@@ -40,7 +40,24 @@ def parse_args():
     ap.add_argument("--workload", default="llava7b_b1")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true",
+                    help="skip the short runs of the other configurations (the `workloads` key)")
+    ap.add_argument("--workload-steps", type=int, default=2)
     return ap.parse_args()
+
+
+def rank_launch_command(gpus, argv, port=None, script=None):
+    """Command line that starts this script as `gpus` ranks on this node (one per GPU, NCCL for
+    the barrier and the max over ranks only): `python bench.py --gpus N` run by hand, with no
+    launcher around it, re-executes itself through torch.distributed.run."""
+    import socket
+    if port is None:
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(gpus),
+            "--master-addr", "127.0.0.1", "--master-port", str(port),
+            os.path.abspath(__file__ if script is None else script)] + list(argv)
 
 
 def measured_peaks():
@@ -104,15 +121,20 @@ class ClockSampler:
         for ln in self.proc.stdout:
             self.lines.append((time.perf_counter(), ln.strip()))
 
-    def stop(self, t0=None, t1=None):
-        """Summary of the samples received in [t0, t1] (host clock), all of them if none fall there."""
+    def stop(self):
         if self.proc is None:
-            return None
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+        self.proc = None
+
+    def window(self, t0=None, t1=None):
+        """Summary of the samples received in [t0, t1] (host clock), all of them if none fall there."""
+        if self.proc is None:
+            return None
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         inside = [ln for ts, ln in self.lines if t0 is None or t0 <= ts <= t1]
@@ -182,22 +204,34 @@ def time_oracle_sample(w, score_layers=1, decode_steps=(0,)):
     return w.B * w.T / total, desc, time.perf_counter() - t_begin
 
 
+def base_config(w):
+    return {"workload": w.name, "batch": w.B, "layers": w.L, "heads": w.H, "head_dim": w.D,
+            "prompt_len": w.N, "budget_rows": w.budget_rows(), "decode_steps": w.T}
+
+
 def run_reference(args):
+    """The oracle, as it stands, on one host core: every step times a bounded sample of the
+    workload (one layer's scoring, compaction and decode, the whole selection) and scales it to
+    the whole step, so `ms_per_step` is an extrapolation and says so."""
     from paper_2412_03409_b200 import workloads as wl
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     w = wl.WORKLOADS[args.workload]
-    vals, desc = [], ""
+    vals, desc, spent = [], "", 0.0
     for i in range(args.warmup + args.steps):
-        v, desc, _ = time_oracle_sample(w)
+        v, desc, sec = time_oracle_sample(w)
         if i >= args.warmup:
             vals.append(v)
+            spent += sec
     value = statistics.mean(vals)
+    cfg = base_config(w)
+    cfg["timing"] = ("each step times a sample (%.2f s of CPU work) and scales it to the whole step: "
+                     "ms_per_step is extrapolated, not elapsed" % (spent / max(1, len(vals))))
     line = {"impl": "reference", "metric": "tok/s", "value": value, "unit": "tok/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.B * w.T / value,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": w.name},
+            "data": "synthetic", "config": cfg,
             "cpu_baseline": {"value": value, "unit": "tok/s", "cores": 1, "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": "tok/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
@@ -206,22 +240,15 @@ def run_reference(args):
 # ---------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------
-def run_ours(args):
+def measure_workload(w, steps, warmup, dev, rank, world, sampler=None, with_lse=False):
+    """Times `steps` passes of the whole path over workload `w` on this rank's samples.
+    Returns per-prompt-batch stage times (ms), algorithmic byte counts and, on request, the
+    scoring time when the caller supplies the log-sum-exp."""
     import torch
-    import torch.distributed as dist
 
-    from paper_2412_03409_b200 import api, sharding, workloads as wl
+    from paper_2412_03409_b200 import sharding, workloads as wl
     from paper_2412_03409_b200.session import Session
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-
-    w = wl.WORKLOADS[args.workload]
     scale = wl.layer_scale(w)
     budget = w.budget_rows()
     # Inputs larger than L2: R independent prompts (replicas) are run interleaved, each as its own
@@ -237,7 +264,6 @@ def run_ours(args):
                     device=dev)
         s.budget.fill_(budget)
         reps.append((s, q, k, v))
-    s, q, k, v = reps[0]
     n_pool = 8
     pool = [wl.make_decode_inputs(w, t, dev, samples=list(range(w.B))) for t in range(n_pool)]
     stream = torch.cuda.current_stream()
@@ -260,57 +286,51 @@ def run_ours(args):
         timed(decode_all, "decode")
 
     def barrier():
+        import torch.distributed as dist
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()                 # nvidia-smi needs a moment to come up: start before warm-up
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step([])
     barrier()
     all_events = []
     wall0 = time.perf_counter()
-    for _ in range(args.steps):
+    for _ in range(steps):
         ev = []
         step(ev)
         all_events.append(ev)
     barrier()
     wall = time.perf_counter() - wall0
-    clocks = sampler.stop(wall0, wall0 + wall) if rank == 0 else None
+    clocks = sampler.window(wall0, wall0 + wall) if sampler is not None else None
     for ss, _, _, _ in reps:
         assert ss.status.cpu().tolist() == [0] * w.B, "device status raised"
 
-    # per prompt: each stage's event time divided by the R prompts it covered
+    # per prompt batch: each stage's event time divided by the R prompts it covered
     stage_ms = {"score": 0.0, "search": 0.0, "compact": 0.0, "decode": 0.0}
     for ev in all_events:
         for tag, a, b in ev:
             stage_ms[tag] += a.elapsed_time(b)
     for kx in stage_ms:
-        stage_ms[kx] /= args.steps * R
-    step_ms = sum(stage_ms.values())
-    step_ms_max = sharding.max_over_ranks(step_ms, dev)
+        stage_ms[kx] /= steps * R
 
+    s0 = reps[0][0]
     # algorithmic bytes of the decode steps (rows actually attended, K and V, plus the append)
-    lens = (s.cache.len.cpu().to(torch.int64) - w.T)      # retained rows after compaction
+    lens = (s0.cache.len.cpu().to(torch.int64) - w.T)      # retained rows after compaction
     retained = int(lens.sum())
-    row_bytes = w.row_bytes
     nseg = w.B * w.L
     io_small = 4 * nseg * w.H * w.D * w.esize             # q, k_new, v_new read + out written
-    dec_bytes = sum(2 * (retained + nseg * (t + 1)) * row_bytes + 2 * nseg * row_bytes + io_small
+    dec_bytes = sum(2 * (retained + nseg * (t + 1)) * w.row_bytes + 2 * nseg * w.row_bytes + io_small
                     for t in range(w.T))
-    dec_gbs = dec_bytes / (stage_ms["decode"] * 1e-3) / 1e9
-    compact_bytes = 2 * 2 * retained * row_bytes
-    compress_ms = stage_ms["score"] + stage_ms["search"] + stage_ms["compact"]
-    causal_flop = 2.0 * w.D * w.N * (w.N + 1) / 2 * w.H * w.L * w.B
-    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    res = {"stage_ms": stage_ms, "R": R, "wall_ms_per_prompt": 1e3 * wall / (steps * R), "clocks": clocks,
+           "dec_bytes": dec_bytes, "compact_bytes": 2 * 2 * retained * w.row_bytes, "budget": budget,
+           "causal_flop": 2.0 * w.D * w.N * (w.N + 1) / 2 * w.H * w.L * w.B, "score_lse_ms": None,
+           "reps": reps, "pool": pool}
 
     # Scoring when the caller's prefill attention kept its log-sum-exp (pass 1 is skipped): timed
     # over the same interleaved prompts, outside the step.  The lse comes from plain torch, untimed.
-    score_lse_ms = None
-    if w.N <= 4096:
+    if with_lse and w.N <= 4096:
         lses = []
         for ss, qq, kk, vv in reps:
             lse = torch.empty((w.B, w.L, w.H, w.N), dtype=torch.float32, device=dev)
@@ -331,13 +351,79 @@ def run_ours(args):
                 ss.score(qq, kk, lse=lse)
         eb.record(stream)
         torch.cuda.synchronize()
-        score_lse_ms = ea.elapsed_time(eb) / (n_rep * R)
+        res["score_lse_ms"] = ea.elapsed_time(eb) / (n_rep * R)
         del lses
+    return res
+
+
+def workload_summary(w, m, hbm_peak, tf_peak):
+    """The figures of one configuration that the targets are stated on."""
+    st = m["stage_ms"]
+    dec_gbs = m["dec_bytes"] / (st["decode"] * 1e-3) / 1e9
+    compress_ms = st["score"] + st["search"] + st["compact"]
+    return {"decode_gbs": dec_gbs, "decode_frac_of_measured_copy": dec_gbs / hbm_peak,
+            "decode_pct_of_8tbs": 100 * dec_gbs / NOMINAL_HBM_GBS, "decode_us_per_call": 1e3 * st["decode"] / w.T,
+            "compress_ms_per_prompt": compress_ms / w.B, "stages_ms": st,
+            "score_tensor_util_vs_burst": m["causal_flop"] * 2 / (st["score"] * 1e-3) / (tf_peak * 1e12),
+            "tok_s": w.B * w.T / (sum(st.values()) * 1e-3), "prompts_interleaved": m["R"], "clocks": m["clocks"]}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2412_03409_b200 import api, sharding, workloads as wl
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # run by hand without a launcher: start the ranks ourselves
+        sys.exit(subprocess.call(rank_launch_command(args.gpus, sys.argv[1:])))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = wl.WORKLOADS[args.workload]
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()                 # nvidia-smi needs a moment to come up: start before warm-up
+    m = measure_workload(w, args.steps, args.warmup, dev, rank, world, sampler if rank == 0 else None,
+                         with_lse=True)
+    stage_ms, R, budget = m["stage_ms"], m["R"], m["budget"]
+    s, q, k, v = m["reps"][0]
+    pool = m["pool"]
+    step_ms = sum(stage_ms.values())
+    step_ms_max = sharding.max_over_ranks(step_ms, dev)
+    dec_bytes = m["dec_bytes"]
+    dec_gbs = dec_bytes / (stage_ms["decode"] * 1e-3) / 1e9
+    compress_ms = stage_ms["score"] + stage_ms["search"] + stage_ms["compact"]
+    hbm_peak, tf_peak, peak_kind = measured_peaks()
+    score_lse_ms = m["score_lse_ms"]
 
     e2e = None
     if not args.no_e2e:
         e2e = run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, max(2, min(args.steps, 5)))
         e2e["ms"] = sharding.max_over_ranks(e2e["ms"], dev)
+    del m["reps"], s, q, k, v
+    torch.cuda.empty_cache()
+
+    # The other configurations, a few steps each (rank 0 of a one-GPU run only): the figures the
+    # bandwidth and latency targets are stated on, measured in this same process.
+    others = {}
+    if world == 1 and not args.no_workloads and args.workload == "llava7b_b1":
+        others[w.name] = workload_summary(w, m, hbm_peak, tf_peak)
+        for name in wl.ORDER:
+            if name == w.name:
+                continue
+            wo = wl.WORKLOADS[name]
+            mo = measure_workload(wo, args.workload_steps, 3, dev, 0, 1, sampler)
+            del mo["reps"], mo["pool"]
+            others[name] = workload_summary(wo, mo, hbm_peak, tf_peak)
+            torch.cuda.empty_cache()
+    clocks = m["clocks"]
+    sampler.stop()
 
     if rank != 0:
         if world > 1:
@@ -349,15 +435,14 @@ def run_ours(args):
         "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.esize == 2 else "f32",
         "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.B, "layers": w.L, "heads": w.H, "head_dim": w.D,
-                   "prompt_len": w.N, "budget_rows": budget, "decode_steps": w.T,
+        "config": {**base_config(w),
                    "parallelism": "batch-sharded x%d, no collective" % world,
                    "prompts_interleaved": R,
                    "l2": "inputs larger than L2: %d independent prompts interleaved call by call, so "
                          ">= 256 MiB of other K/V passes between two calls on one prompt" % R,
                    "timing": "one CUDA-event pair per stage over all %d prompts; ms_per_step and "
                              "stages_ms are per prompt; wall %.2f ms per prompt"
-                             % (R, 1e3 * wall / (args.steps * R))},
+                             % (R, m["wall_ms_per_prompt"])},
         "stages_ms": stage_ms,
         "decode_attn": {"gbs": dec_gbs, "pct_of_8tbs": 100 * dec_gbs / NOMINAL_HBM_GBS,
                         "pct_of_measured_copy": 100 * dec_gbs / hbm_peak,
@@ -365,9 +450,9 @@ def run_ours(args):
         "compress": {"ms_per_prompt": compress_ms / w.B,
                      "ms_per_prompt_given_lse": None if score_lse_ms is None else
                      (score_lse_ms + stage_ms["search"] + stage_ms["compact"]) / w.B,
-                     "compact_gbs": compact_bytes / (stage_ms["compact"] * 1e-3) / 1e9,
-                     "score_tensor_util_vs_burst": causal_flop * 2 / (stage_ms["score"] * 1e-3) / (tf_peak * 1e12),
-                     "target_ms_strict": causal_flop / (0.5 * tf_peak * 1e12) * 1e3},
+                     "compact_gbs": m["compact_bytes"] / (stage_ms["compact"] * 1e-3) / 1e9,
+                     "score_tensor_util_vs_burst": m["causal_flop"] * 2 / (stage_ms["score"] * 1e-3) / (tf_peak * 1e12),
+                     "target_ms_strict": m["causal_flop"] / (0.5 * tf_peak * 1e12) * 1e3},
         "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel + its merge kernel (one decode call, launch gaps included)",
                      "achieved": dec_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": dec_gbs / hbm_peak,
                      "peak_kind": "of " + peak_kind, "traffic": decode_traffic(w.name),
@@ -375,6 +460,8 @@ def run_ours(args):
         "gpu_launches": args.steps * R * LAUNCHES_PER_STEP(w),
         "clocks": clocks,
     }
+    if others:
+        line["workloads"] = others
     if e2e is not None:
         line["e2e"] = {"value": world * w.B * w.T / (e2e["ms"] * 1e-3), "unit": "tok/s",
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
