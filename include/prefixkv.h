@@ -122,15 +122,21 @@ int prefixkv_score(const pkv_shape *shape, const void *q, pkv_strides qs, const 
  * Length rule: p >= 1 keeps N rows; otherwise theta = ceil(p * total) (one fp64
  * multiply) and len = first 1-based j with cum[j-1] >= theta.
  * Search: if L*N <= budget, p = 1.  Else bisect [0,1]: stop when the interval is
- * <= tol wide, after max_iters midpoints, or when fp64 cannot split it; a
- * midpoint whose total S equals the budget, or misses it from below by at most
- * slack_rows, is returned at once; S < budget raises the lower end, otherwise
- * the upper end drops.  On a stop the lower end is returned, so sum(len) never
- * exceeds the budget.
+ * <= tol wide, after max_iters midpoints, or when fp64 cannot split it.  With
+ * delta = S - budget for a midpoint's total S: a midpoint with
+ * -slack_rows <= delta <= slack_over_rows is returned at once (delta = 0 always
+ * is); delta < 0 raises the lower end, otherwise the upper end drops.  On a stop
+ * the lower end is returned, whose total never exceeds the budget.
+ * The two slacks are the threshold on delta of Sec. 3.3 (Tab. "robustness-delta"
+ * states it as a fraction of sum R_l; here it is a number of rows, per side).
+ * slack_over_rows = 0 keeps sum(len) <= budget.  slack_rows = slack_over_rows is
+ * the printed |delta| <= threshold: the configuration may then exceed the budget
+ * by up to that many rows and is to be scaled back with prefixkv_rescale before
+ * prefixkv_compact.
  */
 int prefixkv_search(const pkv_shape *shape, const float *scores, const int64_t *budget_rows,
-                    double tol, int32_t max_iters, int64_t slack_rows, int32_t *order,
-                    uint64_t *cum, int32_t *len, double *p_out, int32_t *iters_out,
+                    double tol, int32_t max_iters, int64_t slack_rows, int64_t slack_over_rows,
+                    int32_t *order, uint64_t *cum, int32_t *len, double *p_out, int32_t *iters_out,
                     int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
@@ -145,12 +151,15 @@ int prefixkv_apply_lengths(const pkv_shape *shape, const float *scores, const in
                            int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
- * Meeting the budget exactly after an inexact search (Sec. 3.3: "scale the resulting global
- * prefix configuration to meet the target budget"; the paper prints no formula).  Reading:
- * every layer keeps its one mandatory row and the other budget - L rows are split in
- * proportion to len - 1 (largest remainder, ties to the lower layer, at most N rows per
- * layer).  A configuration that already sums to its budget is left unchanged; otherwise
- * lengths only grow, so each layer keeps a longer prefix of the same priority sequence.
+ * Meeting the budget exactly after the search (Sec. 3.3 has the configuration found scaled to
+ * the target budget and prints no formula).  Reading: every layer keeps its one mandatory row
+ * and the other budget - L rows are split in proportion to len - 1: floor of the quota first,
+ * at most N rows per layer, then what is left over one row at a time in the order of the
+ * division remainders (largest first, ties to the lower layer), round after round, to the
+ * layers that still have room.  The result sums to min(budget, L*N) exactly.  A configuration
+ * that already sums to its budget is left unchanged; one below it only grows (each layer keeps
+ * a longer prefix of the same priority sequence); one above it -- a search ended by
+ * slack_over_rows -- only shrinks, never below one row per layer.
  *   len          [B,L] int32, in/out (from prefixkv_search)
  *   budget_rows  [B] int64
  * Call it between prefixkv_search and prefixkv_compact.
@@ -192,9 +201,10 @@ typedef struct {
 } pkv_cache;
 
 /*
- * Compression after prefilling (Sec. 3.1; "the top R_l proportion ... retained
- * in each head", Sec. 3.2): for every segment copy the len top-ranked rows of K
- * and V, in ascending prompt position, into the packed cache, and fill
+ * Compression after prefilling (Sec. 3.1; Sec. 3.2: each layer keeps its R_l
+ * highest-ranked vectors, the same set in every head): for every segment copy
+ * the len top-ranked rows of K and V, in ascending prompt position, into the
+ * packed cache, and fill
  * row_offset / len / cap.  Segments whose rows would pass total_cap_rows raise
  * PKV_DEV_CAPACITY and copy nothing.
  *   k, v    [B,L,H,N,D] with strides, as for prefixkv_score
@@ -208,8 +218,8 @@ int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, cons
                      size_t ws_bytes, void *cuda_stream);
 
 /*
- * One decode step over the ragged cache (Sec. 3.1: the newest token "interacts
- * with the cached KV vectors"): for every segment of layers [layer_begin,
+ * One decode step over the ragged cache (Sec. 3.1: the newest token attends over
+ * the cached key/value vectors): for every segment of layers [layer_begin,
  * layer_end), append k_new / v_new as row len, then
  *   out[b,l,h,:] = sum_j softmax_j(scale_l * <q[b,l,h], K_j[h]>) * V_j[h]
  * over all len + 1 rows, and set len += 1.

@@ -114,8 +114,9 @@ class SearchResult:
     status: int
 
 
-def search(cum, budget, tol=1e-6, max_iters=64, slack=0):
-    """Algorithm 1 over cum[L, N] with an integer row budget."""
+def search(cum, budget, tol=1e-6, max_iters=64, slack=0, slack_over=0):
+    """Algorithm 1 over cum[L, N] with an integer row budget.  A midpoint whose total misses the
+    budget by at most `slack` rows from below, or `slack_over` rows from above, ends the search."""
     cum = np.ascontiguousarray(cum, np.uint64)
     L, N = cum.shape
     ln = np.zeros(L, np.int32)
@@ -123,8 +124,8 @@ def search(cum, budget, tol=1e-6, max_iters=64, slack=0):
     it = ctypes.c_int32(0)
     st = _L().orc_search(_p(cum, ctypes.c_uint64), L, N, ctypes.c_int64(int(budget)),
                          ctypes.c_double(float(tol)), ctypes.c_int32(int(max_iters)),
-                         ctypes.c_int64(int(slack)), _p(ln, ctypes.c_int32),
-                         ctypes.byref(p), ctypes.byref(it))
+                         ctypes.c_int64(int(slack)), ctypes.c_int64(int(slack_over)),
+                         _p(ln, ctypes.c_int32), ctypes.byref(p), ctypes.byref(it))
     return SearchResult(ln, p.value, it.value, int(st))
 
 
@@ -175,7 +176,7 @@ def budget_rows(r, L, N):
     return int(np.floor(r * L * N + 1e-9))
 
 
-def select_sample(scores, budget, tol=1e-6, max_iters=64, slack=0):
+def select_sample(scores, budget, tol=1e-6, max_iters=64, slack=0, slack_over=0):
     """Sort + cumulative + search for one sample.  scores: [L, N] fp32."""
     scores = _f32(scores)
     L, N = scores.shape
@@ -189,7 +190,7 @@ def select_sample(scores, budget, tol=1e-6, max_iters=64, slack=0):
     cum = np.stack(cums)
     if status != OK:
         return order, cum, SearchResult(np.zeros(L, np.int32), 0.0, 0, status)
-    return order, cum, search(cum, budget, tol, max_iters, slack)
+    return order, cum, search(cum, budget, tol, max_iters, slack, slack_over)
 
 
 def apportion(weight, budget, N):
@@ -202,7 +203,8 @@ def apportion(weight, budget, N):
 
 
 def rescale(length, budget, N):
-    """Stretch a searched configuration (sum <= budget) to meet the budget exactly."""
+    """Scale a searched configuration to meet the budget exactly (grows one below it, shrinks
+    one above it, never below one row per layer)."""
     return apportion(np.asarray(length, np.int64) - 1, budget, N)
 
 

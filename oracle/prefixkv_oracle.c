@@ -195,15 +195,24 @@ static int64_t total_length(const uint64_t *cum, int L, int N, double p, int32_t
  * loop condition never becomes false, so the search also stops when the
  * interval is no wider than tol, after max_iters evaluations, or when fp64
  * cannot split the interval further; it then returns the lower end p1, whose
- * configuration never exceeds the budget.  A one-sided threshold on delta
- * (0 <= budget - S <= slack) is the paper's "small threshold for delta".
+ * configuration never exceeds the budget.
+ *
+ * Sec. 3.3 also lets the search end as soon as delta is within a small
+ * threshold (Tab. "robustness-delta": the threshold is a fraction of sum R_l,
+ * here a number of rows), after which the configuration is scaled to the
+ * budget.  The threshold is given per side: a midpoint is accepted when
+ *   -slack_under <= delta <= slack_over.
+ * slack_over = 0 never accepts a configuration above the budget; with
+ * slack_under = slack_over the test is the printed |delta| <= threshold, and
+ * the accepted configuration may exceed the budget until it is rescaled
+ * (orc_apportion).
  *
  * cum: [L][N].  Outputs: len[L], *p_out, *iters_out (evaluations of S at a
  * midpoint).  Returns ORC_BUDGET_TOO_SMALL if budget < L.
  * ---------------------------------------------------------------------- */
 int orc_search(const uint64_t *cum, int L, int N, int64_t budget, double tol,
-               int32_t max_iters, int64_t slack, int32_t *len, double *p_out,
-               int32_t *iters_out)
+               int32_t max_iters, int64_t slack_under, int64_t slack_over, int32_t *len,
+               double *p_out, int32_t *iters_out)
 {
     *iters_out = 0;
     if (budget < (int64_t)L) {
@@ -224,7 +233,7 @@ int orc_search(const uint64_t *cum, int L, int N, int64_t budget, double tol,
         int64_t S = total_length(cum, L, N, p, len);
         ++iters;
         int64_t delta = S - budget;
-        if (delta == 0 || (delta < 0 && -delta <= slack)) {
+        if (delta >= -slack_under && delta <= slack_over) {
             *p_out = p;
             *iters_out = iters;
             return ORC_OK;
@@ -323,65 +332,72 @@ double orc_gini(const float *I, const int32_t *order, int N)
 }
 
 /* ------------------------------------------------------------------------
- * Meeting the budget exactly after an inexact search (Sec. 3.3: "scale the
- * resulting global prefix configuration to meet the target budget"; the paper
- * gives no formula) and deriving one configuration from several samples
- * (Sec. 3.3, last paragraph; the aggregation is not specified either).
- * Reading used for both: every layer keeps its one mandatory row; the other
- * budget - L rows are split in proportion to weight[l] (largest-remainder
- * apportionment, ties to the lower layer, at most N rows per layer).
+ * Meeting the budget exactly after the search (Sec. 3.3 says the configuration
+ * found is scaled to the target budget and prints no formula) and deriving one
+ * configuration from several samples (Sec. 3.3, last paragraph; the
+ * aggregation is not specified either).  Reading used for both, an integer
+ * apportionment:
+ *   every layer keeps its one mandatory row; the other E = budget - L rows are
+ *   split in proportion to weight[l]: layer l first gets floor(weight[l] * E / W)
+ *   rows (W = sum of weights), at most N - 1; what is then left over is dealt
+ *   out one row at a time to the layers that still have room, in the order of
+ *   their division remainders (largest first, ties to the lower layer), going
+ *   round as often as needed.
  *   rescale:  weight[l] = len[l] - 1 of the searched configuration
  *   estimate: weight[l] = sum over samples of (len[b][l] - 1)
- * If the searched configuration already sums to the budget it is returned
- * unchanged.  All arithmetic is integer.
+ * Properties: the result sums to min(budget, L * N) exactly; a configuration
+ * that already sums to the budget is returned unchanged; a configuration below
+ * the budget only grows; one above it (a search ended by the two-sided
+ * threshold) only shrinks, never below one row.  All arithmetic is integer.
  * ---------------------------------------------------------------------- */
+typedef struct {
+    int64_t rem;
+    int layer;
+} orc_rem_t;
+
+static int by_remainder(const void *a, const void *b)
+{
+    const orc_rem_t *x = (const orc_rem_t *)a, *y = (const orc_rem_t *)b;
+    if (x->rem != y->rem) return x->rem > y->rem ? -1 : 1;
+    return x->layer < y->layer ? -1 : (x->layer > y->layer ? 1 : 0);
+}
+
 int orc_apportion(const int64_t *weight, int L, int64_t budget, int N, int32_t *len_out)
 {
     if (budget < (int64_t)L) return ORC_BUDGET_TOO_SMALL;
-    int64_t extra = budget - L, cap = (int64_t)N - 1, W = 0;
+    int64_t W = 0;
     for (int l = 0; l < L; ++l) {
         if (weight[l] < 0) return ORC_BAD_LENGTH;
         W += weight[l];
     }
-    int64_t *w = (int64_t *)malloc((size_t)L * sizeof(int64_t));
-    int64_t *x = (int64_t *)malloc((size_t)L * sizeof(int64_t));
-    int64_t *fr = (int64_t *)malloc((size_t)L * sizeof(int64_t));
-    int *ord = (int *)malloc((size_t)L * sizeof(int));
-    for (int l = 0; l < L; ++l) w[l] = W == 0 ? 1 : weight[l];
-    if (W == 0) W = L;
-    int64_t rem = extra;
+    const int64_t E = budget - L, room = (int64_t)N - 1;
+    orc_rem_t *queue = (orc_rem_t *)malloc((size_t)L * sizeof(orc_rem_t));
+    int64_t left = E;
     for (int l = 0; l < L; ++l) {
-        /* w * extra < 2^63 for every supported size (w <= 2^30 rows, extra <= 2^24 rows) */
-        int64_t prod = w[l] * extra;
-        x[l] = prod / W;
-        fr[l] = prod % W;
-        if (x[l] > cap) x[l] = cap;
-        rem -= x[l];
-        ord[l] = l;
+        /* all weights zero: every layer counts the same */
+        const int64_t w = W == 0 ? 1 : weight[l], sum = W == 0 ? L : W;
+        /* w * E < 2^63 for every supported size (w <= 2^30 rows, E <= 2^24 rows) */
+        int64_t share = (w * E) / sum;
+        if (share > room) share = room;
+        len_out[l] = (int32_t)(1 + share);
+        left -= share;
+        queue[l].rem = (w * E) % sum;
+        queue[l].layer = l;
     }
-    /* order: remainder descending, layer ascending (insertion sort, stable) */
-    for (int i = 1; i < L; ++i) {
-        int cur = ord[i], j = i;
-        while (j > 0 && fr[ord[j - 1]] < fr[cur]) {
-            ord[j] = ord[j - 1];
-            --j;
-        }
-        ord[j] = cur;
-    }
-    while (rem > 0) {
-        int given = 0;
-        for (int i = 0; i < L && rem > 0; ++i) {
-            int l = ord[i];
-            if (x[l] < cap) {
-                ++x[l];
-                --rem;
-                ++given;
+    qsort(queue, (size_t)L, sizeof(orc_rem_t), by_remainder);
+    /* one row at a time, round after round, to whoever still has room */
+    while (left > 0) {
+        int64_t before = left;
+        for (int i = 0; i < L && left > 0; ++i) {
+            int l = queue[i].layer;
+            if (len_out[l] < N) {
+                len_out[l] += 1;
+                left -= 1;
             }
         }
-        if (!given) break; /* every layer already keeps all N rows */
+        if (left == before) break; /* every layer already keeps all N rows */
     }
-    for (int l = 0; l < L; ++l) len_out[l] = (int32_t)(1 + x[l]);
-    free(w); free(x); free(fr); free(ord);
+    free(queue);
     return ORC_OK;
 }
 

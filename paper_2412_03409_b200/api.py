@@ -65,7 +65,7 @@ def _load():
                              ctypes.c_size_t)
     sp = ctypes.POINTER(Shape)
     lib.prefixkv_score.argtypes = [sp, vp, Strides, vp, Strides, vp, vp, vp, vp, sz, vp]
-    lib.prefixkv_search.argtypes = [sp, vp, vp, f64, i32, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.prefixkv_search.argtypes = [sp, vp, vp, f64, i32, i64, i64, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.prefixkv_apply_lengths.argtypes = [sp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.prefixkv_compact.argtypes = [sp, vp, Strides, vp, Strides, vp, vp,
                                      ctypes.POINTER(CacheStruct), vp, vp, vp, sz, vp]
@@ -137,10 +137,10 @@ def prefixkv_score(shape, q, k, layer_scale, scores, ws, lse=None):
 
 
 def prefixkv_search(shape, scores, budget_rows, tol, max_iters, slack_rows, order, cum, length,
-                    p_out, iters_out, dev_status, ws=None):
+                    p_out, iters_out, dev_status, ws=None, slack_over_rows=0):
     p, n = _ws(ws)
     _check(_lib.prefixkv_search(ctypes.byref(shape), _ptr(scores), _ptr(budget_rows), float(tol),
-                                int(max_iters), int(slack_rows), _ptr(order), _ptr(cum),
+                                int(max_iters), int(slack_rows), int(slack_over_rows), _ptr(order), _ptr(cum),
                                 _ptr(length), _ptr(p_out), _ptr(iters_out), _ptr(dev_status), p, n,
                                 _stream()), "prefixkv_search")
 

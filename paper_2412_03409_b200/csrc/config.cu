@@ -1,11 +1,14 @@
-// Exact budget and offline configuration (Sec. 3.3).  The paper says to "scale the resulting
-// global prefix configuration to meet the target budget" after an inexact search, and to
-// derive one configuration from a few sample prompts, without giving either formula.  Both
-// are done here by one integer apportionment: every layer keeps its one mandatory row and
-// the other budget - L rows are split in proportion to a weight per layer (largest remainder,
-// ties to the lower layer, at most N rows per layer):
+// Exact budget and offline configuration (Sec. 3.3).  After the search the paper has the
+// configuration scaled to the target budget, and it derives one configuration from a few sample
+// prompts, without giving either formula.  Both are done here by one integer apportionment:
+// every layer keeps its one mandatory row and the other budget - L rows are split in
+// proportion to a weight per layer -- the floor of the quota first (at most N rows per layer),
+// then what is left over one row at a time in the order of the division remainders (largest
+// first, ties to the lower layer), round after round, to the layers that still have room:
 //   rescale:  weight[l] = len[b][l] - 1 of sample b's searched configuration
 //   estimate: weight[l] = sum over the sample prompts of (len[k][l] - 1)
+// A configuration above its budget (a search ended by the threshold on the upper side) comes
+// out shorter, never below one row per layer; one below it comes out longer.
 #include "common.cuh"
 
 namespace pkv {
@@ -26,13 +29,17 @@ __device__ __forceinline__ int64_t block_sum_i64(int64_t v, int64_t *red)
 }
 
 // One CTA per problem; thread l owns layer l.  `samples` rows of len_in are summed per problem.
+// The left-over rows are dealt in whole rounds, all layers in parallel: while more rows are left
+// than layers have room, every open layer takes min(rows left / open layers, its room) at once
+// (what going round one row at a time would have given it by then); the last, partial round
+// goes to the first `left` open layers in remainder order.
 __global__ void __launch_bounds__(kMaxLayers)
 apportion_kernel(const int32_t *len_in, int samples, int L, int N, const int64_t *budget_dev,
                  int64_t budget_host, int32_t *len_out, int32_t *dev_status)
 {
     __shared__ int64_t red[32];
-    __shared__ int64_t s_fr[kMaxLayers];
-    __shared__ int s_x[kMaxLayers], s_order[kMaxLayers];
+    __shared__ int64_t s_rem[kMaxLayers];
+    __shared__ unsigned char s_open[kMaxLayers];  // by rank in remainder order: has the layer room?
     const int p = blockIdx.x, l = threadIdx.x;
     const bool mine = l < L;
     const int64_t budget = budget_dev ? budget_dev[p] : budget_host;
@@ -55,43 +62,45 @@ apportion_kernel(const int32_t *len_in, int samples, int L, int N, const int64_t
         return;
     }
     int64_t W = block_sum_i64(w, red);
-    if (W == 0) {
+    if (W == 0) {  // all weights zero: every layer counts the same
         w = mine ? 1 : 0;
         W = L;
     }
-    const int64_t extra = budget - L, cap = (int64_t)N - 1;
+    const int64_t extra = budget - L, room0 = (int64_t)N - 1;
     const int64_t prod = w * extra;  // < 2^63: w <= 2^30 rows, extra <= 2^24 rows for supported sizes
     int64_t x = prod / W;
-    const int64_t fr = prod % W;
-    if (x > cap) x = cap;
-    if (mine) {
-        s_fr[l] = fr;
-        s_x[l] = (int)x;
-    }
-    int64_t rem = extra - block_sum_i64(mine ? x : 0, red);
-    // rank by (remainder descending, layer ascending)
-    if (mine) {
-        int rank = 0;
-        for (int j = 0; j < L; ++j) rank += (s_fr[j] > fr) || (s_fr[j] == fr && j < l);
-        s_order[rank] = l;
-    }
-    __syncthreads();
-    if (l == 0) {
-        while (rem > 0) {
-            int given = 0;
-            for (int i = 0; i < L && rem > 0; ++i) {
-                const int ll = s_order[i];
-                if (s_x[ll] < cap) {
-                    ++s_x[ll];
-                    --rem;
-                    ++given;
-                }
-            }
-            if (!given) break;  // every layer already keeps all N rows
+    const int64_t rem = prod % W;
+    if (x > room0) x = room0;
+    if (mine) s_rem[l] = rem;
+    int64_t left = extra - block_sum_i64(mine ? x : 0, red);
+    // this layer's place in the order (remainder descending, layer ascending)
+    int rank = 0;
+    if (mine)
+        for (int j = 0; j < L; ++j) rank += (s_rem[j] > rem) || (s_rem[j] == rem && j < l);
+    for (;;) {  // uniform over the CTA: `left` and the counts below are block-wide sums
+        const int64_t room = mine ? room0 - x : 0;
+        const int64_t open = block_sum_i64(room > 0 ? 1 : 0, red);
+        if (left <= 0 || open == 0) break;
+        if (left >= open) {
+            // whole rounds: every open layer takes one row per round until it is full or the
+            // rounds that all currently open layers can share are over
+            const int64_t rounds = left / open;
+            const int64_t take = room < rounds ? room : rounds;
+            x += take;
+            left -= block_sum_i64(take, red);
+        } else {
+            // the last round reaches only the first `left` open layers of the order
+            if (mine) s_open[rank] = room > 0;
+            __syncthreads();
+            int ahead = 0;  // open layers before this one in the order
+            if (mine && room > 0)
+                for (int r = 0; r < rank; ++r) ahead += s_open[r];
+            if (mine && room > 0 && ahead < left) x += 1;
+            left = 0;
+            break;
         }
     }
-    __syncthreads();
-    if (mine) len_out[(size_t)p * L + l] = 1 + s_x[l];
+    if (mine) len_out[(size_t)p * L + l] = (int32_t)(1 + x);
 }
 
 static int threads_for(int L)

@@ -187,7 +187,7 @@ __device__ __forceinline__ int warp_length_for_theta(const uint64_t *__restrict_
 // that one barrier per midpoint is enough.
 __global__ void __launch_bounds__(1024)
 search_kernel(const uint64_t *__restrict__ cum, const int64_t *__restrict__ budget_rows, int L,
-              int N, double tol, int max_iters, int64_t slack, int32_t *__restrict__ len,
+              int N, double tol, int max_iters, int64_t slack, int64_t slack_over, int32_t *__restrict__ len,
               double *__restrict__ p_out, int32_t *__restrict__ iters_out, int32_t *dev_status)
 {
     extern __shared__ int s_len[];  // [2][L]
@@ -270,7 +270,7 @@ search_kernel(const uint64_t *__restrict__ cum, const int64_t *__restrict__ budg
             int64_t S = eval(p, buf);
             ++iters;
             int64_t delta = S - budget;
-            if (delta == 0 || (delta < 0 && -delta <= slack)) {
+            if (delta >= -slack && delta <= slack_over) {  // within the threshold on delta (Sec. 3.3)
                 p_final = p;
                 have = true;
                 break;
@@ -336,13 +336,13 @@ using namespace pkv;
 
 extern "C" int prefixkv_search(const pkv_shape *shape, const float *scores,
                                const int64_t *budget_rows, double tol, int32_t max_iters,
-                               int64_t slack_rows, int32_t *order, uint64_t *cum, int32_t *len,
-                               double *p_out, int32_t *iters_out, int32_t *dev_status, void *ws,
-                               size_t ws_bytes, void *cuda_stream)
+                               int64_t slack_rows, int64_t slack_over_rows, int32_t *order, uint64_t *cum,
+                               int32_t *len, double *p_out, int32_t *iters_out, int32_t *dev_status,
+                               void *ws, size_t ws_bytes, void *cuda_stream)
 {
     (void)ws; (void)ws_bytes;
     if (!shape_ok(shape) || !scores || !budget_rows || !order || !cum || !len || !p_out ||
-        !iters_out || !dev_status || !(tol >= 0.0) || max_iters < 0 || slack_rows < 0)
+        !iters_out || !dev_status || !(tol >= 0.0) || max_iters < 0 || slack_rows < 0 || slack_over_rows < 0)
         return PKV_ERR_INVALID_ARG;
     if (!shape_supported(shape)) return PKV_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
@@ -352,7 +352,7 @@ extern "C" int prefixkv_search(const pkv_shape *shape, const float *scores,
     int rc = launch_sort(shape, scores, order, cum, dev_status, st);
     if (rc != PKV_OK) return rc;
     cudaError_t e = launch_dependent(search_kernel, dim3(B), dim3(1024), 2 * L * sizeof(int), st,
-                                     (const uint64_t *)cum, budget_rows, L, N, tol, (int)max_iters, slack_rows, len,
+                                     (const uint64_t *)cum, budget_rows, L, N, tol, (int)max_iters, slack_rows, slack_over_rows, len,
                                      p_out, iters_out, dev_status);
     if (e != cudaSuccess) {
         set_cuda_error(e, "search_kernel");

@@ -44,14 +44,14 @@ class Session:
         api.prefixkv_score(self.shape, q, k, self.layer_scale, self.scores, self.ws_score, lse=lse)
         return self.scores
 
-    def search(self, budget_rows, tol=1e-6, max_iters=64, slack_rows=0, scores=None):
+    def search(self, budget_rows, tol=1e-6, max_iters=64, slack_rows=0, scores=None, slack_over_rows=0):
         if isinstance(budget_rows, torch.Tensor):
             self.budget.copy_(budget_rows)
         elif budget_rows is not None:          # None: keep the budget already on the device
             self.budget.fill_(int(budget_rows))
         api.prefixkv_search(self.shape, self.scores if scores is None else scores, self.budget, tol,
                             max_iters, slack_rows, self.order, self.cum, self.len, self.p,
-                            self.iters, self.status)
+                            self.iters, self.status, slack_over_rows=slack_over_rows)
 
     def apply_lengths(self, len_in, scores=None):
         len_in = len_in.to(self.device, torch.int32).contiguous()

@@ -56,11 +56,11 @@ def test_null_and_range_arguments_rejected_on_host(api):
     sh = api.make_shape(1, 2, 4, 64, 32, torch.float32)
     z = api.Strides(0, 0, 0, 0)
     assert lib.prefixkv_score(sh, None, z, None, z, None, None, None, None, 0, None) == api.PKV_ERR_INVALID_ARG
-    assert lib.prefixkv_search(sh, None, None, 1e-6, 64, 0, None, None, None, None, None, None,
+    assert lib.prefixkv_search(sh, None, None, 1e-6, 64, 0, 0, None, None, None, None, None, None,
                                None, 0, None) == api.PKV_ERR_INVALID_ARG
     if torch.cuda.is_available():
         return      # the cases below pass made-up non-null addresses: only where no launch can reach a GPU
-    assert lib.prefixkv_search(sh, 16, 16, -1.0, 64, 0, 16, 16, 16, 16, 16, 16, None, 0, None) == \
+    assert lib.prefixkv_search(sh, 16, 16, -1.0, 64, 0, 0, 16, 16, 16, 16, 16, 16, None, 0, None) == \
         api.PKV_ERR_INVALID_ARG                                    # negative tolerance
     assert lib.prefixkv_apply_lengths(sh, None, None, 0, None, None, None, None, None, 0, None) == \
         api.PKV_ERR_INVALID_ARG

@@ -65,6 +65,59 @@ def test_selection_slack_and_iteration_cap(api):
         assert s.p[0].item() == res.p and s.iters[0].item() == res.iters
 
 
+@pytest.mark.parametrize("B,L,N", [(3, 8, 300), (2, 32, 640)])
+def test_selection_two_sided_threshold_then_rescale(api, B, L, N):
+    """Sec. 3.3: the search ends once |delta| is within a threshold (per side here), possibly above
+    the budget; prefixkv_rescale then meets the budget exactly.  Both bit for bit against the oracle."""
+    scores = np.stack([wl.synthetic_scores(L, N, seed=b + 40) for b in range(B)])
+    budgets = [L * N // 3 + 11 * b for b in range(B)]
+    over_seen = False
+    for under, over in [(0, 3), (5, 5), (0, 25), (40, 40), (L * N, L * N)]:
+        s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+        s.search(torch.tensor(budgets), tol=0.0, max_iters=2000, slack_rows=under, slack_over_rows=over,
+                 scores=torch.from_numpy(scores).cuda())
+        searched = s.len.cpu().numpy().copy()
+        api.prefixkv_rescale(s.shape, s.len, s.budget, s.status)
+        fixed = s.len.cpu().numpy()
+        for b in range(B):
+            _, _, res = oracle.select_sample(scores[b], budgets[b], 0.0, 2000, under, over)
+            np.testing.assert_array_equal(searched[b], res.len)
+            assert s.p[b].item() == res.p and s.iters[b].item() == res.iters
+            assert -under <= int(res.len.sum()) - budgets[b] <= over or res.iters > 30
+            ref, st = oracle.rescale(res.len, budgets[b], N)
+            assert st == oracle.OK
+            np.testing.assert_array_equal(fixed[b], ref)
+            assert fixed[b].sum() == budgets[b] and (fixed[b] >= 1).all()
+            if res.len.sum() > budgets[b]:
+                over_seen = True
+                assert (fixed[b] <= res.len).all()
+        assert s.status.cpu().tolist() == [0] * B
+    assert over_seen                                  # some search did end above its budget
+
+
+def test_rescale_with_full_layers(api):
+    """Budgets close to L * N: layers reach all N rows and what they cannot take goes round to the
+    others (many rounds for the kernel's bulk hand-out to reproduce)."""
+    rng = np.random.default_rng(8)
+    B, L, N = 8, 40, 64
+    lens = rng.integers(1, N + 1, (B, L)).astype(np.int32)
+    lens[0] = 1                                          # all weights zero
+    lens[1, :35] = N                                     # most layers already full
+    budgets = np.array([L * N - 3, L * N - 40, L * N, L * N + 9, L * N // 2, L, L + 1, L * N - 700])
+    s = _session(B, L, 4, 64, N, torch.float32, np.ones(L), decode_cap=1)
+    s.len.copy_(torch.from_numpy(lens))
+    s.budget.copy_(torch.from_numpy(budgets))
+    s.status.zero_()
+    api.prefixkv_rescale(s.shape, s.len, s.budget, s.status)
+    got = s.len.cpu().numpy()
+    for b in range(B):
+        ref, st = oracle.rescale(lens[b], int(budgets[b]), N)
+        assert st == oracle.OK
+        np.testing.assert_array_equal(got[b], ref)
+        assert got[b].sum() == min(int(budgets[b]), L * N)
+    assert s.status.cpu().tolist() == [0] * B
+
+
 def test_selection_degenerate_cases(api):
     L, N = 4, 64
     scores = wl.synthetic_scores(L, N, seed=9)
@@ -510,7 +563,7 @@ def test_argument_validation_fails_on_the_host(api):
     s.len.fill_(-5)
     s.status.fill_(0)
     p = lambda t: t.data_ptr()
-    rc = api.lib().prefixkv_search(bad, p(s.scores), p(s.budget), 0.0, 1, 0, p(s.order), p(s.cum), p(s.len),
+    rc = api.lib().prefixkv_search(bad, p(s.scores), p(s.budget), 0.0, 1, 0, 0, p(s.order), p(s.cum), p(s.len),
                                    p(s.p), p(s.iters), p(s.status), None, 0, None)
     torch.cuda.synchronize()
     assert rc == api.PKV_ERR_UNSUPPORTED

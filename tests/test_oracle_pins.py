@@ -427,45 +427,124 @@ def test_gini_closed_forms():
 # Meeting the budget exactly / offline configuration (Sec. 3.3)
 # --------------------------------------------------------------------------
 def _hamilton(weight, budget, N):
-    """Largest-remainder apportionment with exact rationals (independent of the oracle)."""
+    """Hamilton's largest-remainder apportionment in closed form with exact rationals: every layer
+    gets the floor of its quota, and the layers with the `rem` largest fractional parts (ties to
+    the lower layer) one more -- one round, because fewer than L rows are left after the floors.
+    Returns None when a layer would pass N rows (the cap is outside this textbook form)."""
     L = len(weight)
-    extra, cap = budget - L, N - 1
+    extra = budget - L
     w = [int(x) for x in weight]
     if sum(w) == 0:
         w = [1] * L
     W = sum(w)
     quota = [Fraction(x * extra, W) for x in w]
-    x = [min(cap, q.numerator // q.denominator) for q in quota]
-    order = sorted(range(L), key=lambda l: (-(quota[l] - (quota[l].numerator // quota[l].denominator)), l))
-    rem = extra - sum(x)
-    while rem > 0:
-        given = 0
-        for l in order:
-            if rem > 0 and x[l] < cap:
-                x[l] += 1; rem -= 1; given += 1
-        if not given:
-            break
-    return [1 + v for v in x]
+    floors = [q.numerator // q.denominator for q in quota]
+    rem = extra - sum(floors)
+    assert 0 <= rem < L
+    lucky = sorted(range(L), key=lambda l: (-(quota[l] - floors[l]), l))[:rem]
+    out = [1 + floors[l] + (1 if l in lucky else 0) for l in range(L)]
+    return out if max(out) <= N else None
 
 
 def test_rescale_meets_budget_and_keeps_proportions():
     rng = np.random.default_rng(21)
-    for _ in range(40):
+    uncapped = capped = shrunk = 0
+    for _ in range(120):
         L, N = int(rng.integers(1, 12)), int(rng.integers(2, 60))
         length = rng.integers(1, N + 1, L)
-        budget = int(rng.integers(length.sum(), L * N + 5))
+        budget = int(rng.integers(L, L * N + 5))
         out, st = oracle.rescale(length, budget, N)
         assert st == oracle.OK
         assert out.sum() == min(budget, L * N)
-        assert (out >= length).all() and (out <= N).all() and (out >= 1).all()
-        assert list(out) == _hamilton(length - 1, budget, N)
+        assert (out <= N).all() and (out >= 1).all()
+        if budget >= length.sum():
+            assert (out >= length).all()                   # a configuration below the budget only grows
+        else:
+            assert (out <= length).all()                   # one above it only shrinks, never below one row
+            shrunk += 1
+        ref = _hamilton(length - 1, budget, N)
+        if ref is not None:
+            assert list(out) == ref
+            uncapped += 1
+        else:
+            # the cap binds: whoever is not full got at least its floor quota, and a layer with a
+            # larger weight never ends up with fewer rows
+            capped += 1
+            w = length - 1
+            for a in range(L):
+                for b in range(L):
+                    if w[a] > w[b]:
+                        assert out[a] >= out[b]
         same, _ = oracle.rescale(length, int(length.sum()), N)      # nothing to do: unchanged
         np.testing.assert_array_equal(same, length)
+    assert uncapped > 20 and capped > 5 and shrunk > 20
     # the hand-worked search example: budget 4 was missed by one row (len = (1, 2)); the row
     # goes to the layer with the larger share beyond its mandatory row
     out, _ = oracle.rescale([1, 2], 4, 3)
     assert list(out) == [1, 3]
     assert oracle.rescale([1, 2], 1, 3)[1] == oracle.BUDGET_TOO_SMALL
+
+
+def _bisect_model(cum, budget, under, over, max_iters=4000):
+    """Algorithm 1 retold with Python integers and the independent length rule above: the
+    midpoints are k / 2^j, the first one whose total lies within the thresholds is the answer."""
+    L = cum.shape[0]
+    lo, hi, it = Fraction(0), Fraction(1), 0
+    while it < max_iters:
+        mid = (lo + hi) / 2
+        if float(mid) in (float(lo), float(hi)):
+            break
+        S = sum(_length_exact(cum[l], float(mid)) for l in range(L))
+        it += 1
+        if -under <= S - budget <= over:
+            return float(mid), it, S
+        if S < budget:
+            lo = mid
+        else:
+            hi = mid
+    return float(lo), it, sum(_length_exact(cum[l], float(lo)) for l in range(L))
+
+
+@pytest.mark.parametrize("seed", range(5))
+def test_search_two_sided_threshold(seed):
+    """Sec. 3.3 / Tab. robustness-delta: the search may end once |delta| is within a threshold;
+    the configuration is then scaled to the budget."""
+    rng = np.random.default_rng(300 + seed)
+    L, N = int(rng.integers(3, 8)), int(rng.integers(20, 60))
+    scores = np.exp(rng.standard_normal((L, N)) * rng.uniform(0.3, 2.0, (L, 1))).astype(np.float32)
+    budget = L * N // 3
+    prev_iters = None
+    for delta in (0, 1, 2, 4, 8, 16, 40):
+        _, cum, res = oracle.select_sample(scores, budget, tol=0.0, max_iters=4000, slack=delta, slack_over=delta)
+        p_ref, it_ref, S_ref = _bisect_model(cum, budget, delta, delta)
+        assert (res.p, res.iters, int(res.len.sum())) == (p_ref, it_ref, S_ref)
+        if prev_iters is not None:
+            assert res.iters <= prev_iters                 # a wider threshold never needs more steps
+        prev_iters = res.iters
+        fixed, st = oracle.rescale(res.len, budget, N)     # "scale ... to meet the target budget"
+        assert st == oracle.OK and fixed.sum() == budget and (fixed >= 1).all() and (fixed <= N).all()
+        if res.len.sum() > budget:
+            assert (fixed <= res.len).all()
+        # over-side only: never accepted below the budget unless exact
+        _, _, ro = oracle.select_sample(scores, budget, tol=0.0, max_iters=4000, slack=0, slack_over=delta)
+        assert (ro.p, ro.iters) == _bisect_model(cum, budget, 0, delta)[:2]
+    # a threshold as wide as the whole range accepts the very first midpoint
+    _, _, r1 = oracle.select_sample(scores, budget, slack=L * N, slack_over=L * N)
+    assert r1.iters == 1 and r1.p == 0.5
+
+
+def test_search_delta_hand_example():
+    A = np.array([11, 3, 2], np.float32) / 16
+    B = np.array([6, 5, 5], np.float32) / 16
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "search_delta_hand_example.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 5
+    for budget, under, over, p, la, lb, steps, ra, rb in rows:
+        _, _, res = oracle.select_sample(np.stack([A, B]), int(budget), tol=0.0, max_iters=4000,
+                                         slack=int(under), slack_over=int(over))
+        assert (res.p, list(res.len), res.iters) == (float(p), [int(la), int(lb)], int(steps))
+        fixed, _ = oracle.rescale(res.len, int(budget), 3)
+        assert list(fixed) == [int(ra), int(rb)] and fixed.sum() == int(budget)
 
 
 def test_offline_configuration_from_samples():
