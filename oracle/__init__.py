@@ -153,6 +153,34 @@ def gather_rows(src, kept):
     return dst
 
 
+MERGE_POSITION, MERGE_FEATURE = 1, 2
+
+
+def merge_match(k, kept, mode, want_gap=False):
+    """Which retained vector every position merges into (Sec. 4.3).  k [H, N, D]; kept ascending.
+    Returns match[H, N] (indices into kept) and, on request, the best-minus-second metric."""
+    k = _f32(k)
+    kept = np.ascontiguousarray(kept, np.int32)
+    H, N, D = k.shape
+    match = np.empty((H, N), np.int32)
+    gap = np.empty((H, N), np.float64)
+    _L().orc_merge_match(_p(k, ctypes.c_float), H, N, D, _p(kept, ctypes.c_int32), kept.shape[0], int(mode),
+                         _p(match, ctypes.c_int32), _p(gap, ctypes.c_double))
+    return (match, gap) if want_gap else match
+
+
+def merge_rows(src, kept, match):
+    """Merged cache rows [len, H, D] (fp64) of src [H, N, D] under the assignment match[H, N]."""
+    src = _f32(src)
+    kept = np.ascontiguousarray(kept, np.int32)
+    match = np.ascontiguousarray(match, np.int32)
+    H, N, D = src.shape
+    dst = np.empty((kept.shape[0], H, D), np.float64)
+    _L().orc_merge_rows(_p(src, ctypes.c_float), H, N, D, _p(kept, ctypes.c_int32), kept.shape[0],
+                        _p(match, ctypes.c_int32), _p(dst, ctypes.c_double))
+    return dst
+
+
 def decode_attn(q, kc, vc, scale):
     """q [H, D]; kc, vc [rows, H, D] (new row already appended) -> [H, D] fp64."""
     q, kc, vc = _f32(q), _f32(kc), _f32(vc)

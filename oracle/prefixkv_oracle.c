@@ -19,7 +19,8 @@
  * the closed form log(m) for zero queries for the normaliser; library stable sort for the
  * order; exact rational arithmetic for the cumulative weights; brute-force
  * enumeration of every breakpoint of p and a hand-worked example for the
- * search; library dense attention for decode.  Unpinned: nothing in this file
+ * search; library dense attention for decode; a hand example, one-hot keys
+ * and a library normalised matrix product for cache merging.  Unpinned: nothing in this file
  * (iteration counts and model quality reported by the paper are not
  * reproducible without its data and are not claimed).
  */
@@ -280,6 +281,96 @@ void orc_gather_rows(const float *src, int H, int N, int D, const int32_t *kept,
         for (int h = 0; h < H; ++h)
             memcpy(dst + ((size_t)r * H + h) * D,
                    src + ((size_t)h * N + kept[r]) * D, (size_t)D * sizeof(float));
+}
+
+/* ------------------------------------------------------------------------
+ * Cache merging, Sec. 4.3 ("Eviction or merging", Tab. "merge"): instead of
+ * being dropped, every pruned vector is merged into one retained vector.  With
+ * Omega_r the retained positions (kept[], ascending) and Omega_p the others,
+ * each pruned key k^m is matched to the retained key with the largest metric
+ *   Position:  c^{mn} = -|m - n|
+ *   Feature:   c^{mn} = (k^m . k^n) / (|k^m| |k^n|)     (0 when a norm is 0)
+ * T^n collects the pruned positions matched to n, and the retained vector is
+ * replaced by the plain average of itself and the vectors in T^n.  The
+ * operation is done per head and is the same for keys and values.
+ * Readings (the paper is silent): the match is taken on the keys and applied to
+ * the values as well; among equal metrics the retained vector at the lower
+ * position wins.
+ *
+ * orc_merge_match: k [H][N][D]; match[H][N] receives, for every position, the
+ * index r into kept[] it belongs to (its own index for a retained position).
+ * gap[H][N] (may be NULL) receives best minus second-best metric of a pruned
+ * position (+inf when only one candidate), so that a test can tell a real
+ * decision from a near tie.  mode: 1 = Position, 2 = Feature.
+ * ---------------------------------------------------------------------- */
+void orc_merge_match(const float *k, int H, int N, int D, const int32_t *kept, int32_t len,
+                     int mode, int32_t *match, double *gap)
+{
+    int32_t *slot = (int32_t *)malloc((size_t)N * sizeof(int32_t));
+    for (int n = 0; n < N; ++n) slot[n] = -1;
+    for (int r = 0; r < len; ++r) slot[kept[r]] = r;
+    for (int h = 0; h < H; ++h) {
+        const float *kh = k + (size_t)h * N * D;
+        for (int m = 0; m < N; ++m) {
+            int32_t *out = match + (size_t)h * N + m;
+            if (slot[m] >= 0) {
+                *out = slot[m];
+                if (gap) gap[(size_t)h * N + m] = INFINITY;
+                continue;
+            }
+            double best = -INFINITY, second = -INFINITY;
+            int32_t arg = -1;
+            double nm = 0.0;
+            for (int d = 0; d < D; ++d) nm += (double)kh[(size_t)m * D + d] * (double)kh[(size_t)m * D + d];
+            for (int r = 0; r < len; ++r) {
+                const int n = kept[r];
+                double c;
+                if (mode == 1) {
+                    c = -fabs((double)m - (double)n);
+                } else {
+                    double dot = 0.0, nn = 0.0;
+                    for (int d = 0; d < D; ++d) {
+                        dot += (double)kh[(size_t)m * D + d] * (double)kh[(size_t)n * D + d];
+                        nn += (double)kh[(size_t)n * D + d] * (double)kh[(size_t)n * D + d];
+                    }
+                    c = (nm > 0.0 && nn > 0.0) ? dot / (sqrt(nm) * sqrt(nn)) : 0.0;
+                }
+                if (c > best) { /* strict: an equal metric later in kept[] (a higher position) loses */
+                    second = best;
+                    best = c;
+                    arg = r;
+                } else if (c > second) {
+                    second = c;
+                }
+            }
+            *out = arg;
+            if (gap) gap[(size_t)h * N + m] = best - second;
+        }
+    }
+    free(slot);
+}
+
+/* The merged cache rows for a given assignment: dst[r][h][:] = average of src[h][kept[r]][:] and
+ * of every src[h][m][:] with match[h][m] == r, m not retained.  src [H][N][D]; dst [len][H][D]. */
+void orc_merge_rows(const float *src, int H, int N, int D, const int32_t *kept, int32_t len,
+                    const int32_t *match, double *dst)
+{
+    int32_t *count = (int32_t *)malloc((size_t)len * sizeof(int32_t));
+    for (int h = 0; h < H; ++h) {
+        for (int r = 0; r < len; ++r) {
+            count[r] = 0;
+            for (int d = 0; d < D; ++d) dst[((size_t)r * H + h) * D + d] = 0.0;
+        }
+        for (int m = 0; m < N; ++m) {
+            const int32_t r = match[(size_t)h * N + m];
+            count[r] += 1; /* the retained vector itself is listed under its own index */
+            for (int d = 0; d < D; ++d)
+                dst[((size_t)r * H + h) * D + d] += (double)src[((size_t)h * N + m) * D + d];
+        }
+        for (int r = 0; r < len; ++r)
+            for (int d = 0; d < D; ++d) dst[((size_t)r * H + h) * D + d] /= (double)count[r];
+    }
+    free(count);
 }
 
 /* ------------------------------------------------------------------------

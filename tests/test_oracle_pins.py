@@ -611,3 +611,72 @@ def test_decode_time_pruning_rule(len0, N, d):
         assert n == len0 + steps                                                            # nothing dropped
     else:
         assert n < len0 + steps
+
+
+# --------------------------------------------------------------------------
+# Cache merging (Sec. 4.3, "Eviction or merging")
+# --------------------------------------------------------------------------
+def test_merge_position_hand_example():
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "merge_position_hand_example.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    N = int(rows[0][0])
+    kept = np.array([int(x) for x in rows[1]], np.int32)
+    want_match = [int(x) for x in rows[2]]
+    want_rows = [float(x) for x in rows[3]]
+    src = np.arange(N, dtype=np.float32)[None, :, None] * np.ones((2, 1, 3), np.float32)   # k[h, p, :] = p
+    match = oracle.merge_match(src, kept, oracle.MERGE_POSITION)
+    assert match[0].tolist() == want_match and match[1].tolist() == want_match
+    merged = oracle.merge_rows(src, kept, match)
+    np.testing.assert_allclose(merged[:, 0, 0], want_rows, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(merged[:, 1, 2], want_rows, rtol=0, atol=1e-12)
+
+
+def test_merge_feature_special_cases_and_library():
+    rng = np.random.default_rng(31)
+    H, N, D = 3, 40, 8
+    # one-hot keys: a pruned key merges into the retained key with the same hot index
+    hot = rng.integers(0, D, (H, N))
+    k = np.zeros((H, N, D), np.float32)
+    for h in range(H):
+        k[h, np.arange(N), hot[h]] = rng.uniform(0.5, 2.0, N).astype(np.float32)
+    kept = np.sort(rng.choice(N, 14, replace=False)).astype(np.int32)
+    match = oracle.merge_match(k, kept, oracle.MERGE_FEATURE)
+    for h in range(H):
+        for m in range(N):
+            same = [r for r, n in enumerate(kept) if hot[h, n] == hot[h, m]]
+            if m in kept:
+                assert kept[match[h, m]] == m
+            elif same:
+                assert match[h, m] == same[0]              # the lowest position among equal cosines (all 1)
+            else:
+                assert match[h, m] == 0                    # every cosine is 0: the lowest retained position
+    # random keys: a normalised matrix product and argmax from the library
+    k = rng.standard_normal((H, N, D)).astype(np.float32)
+    v = rng.standard_normal((H, N, D)).astype(np.float32)
+    match, gap = oracle.merge_match(k, kept, oracle.MERGE_FEATURE, want_gap=True)
+    kn = k.astype(np.float64) / np.linalg.norm(k.astype(np.float64), axis=-1, keepdims=True)
+    cos = np.einsum("hmd,hnd->hmn", kn, kn[:, kept])
+    pruned = np.setdiff1d(np.arange(N), kept)
+    np.testing.assert_array_equal(match[:, pruned], cos.argmax(axis=-1)[:, pruned])
+    top2 = np.sort(cos, axis=-1)[:, :, -2:]
+    np.testing.assert_allclose(gap[:, pruned], (top2[..., 1] - top2[..., 0])[:, pruned], atol=1e-12)
+    # merged rows: scatter-add with numpy, and the total is preserved
+    merged = oracle.merge_rows(v, kept, match)
+    acc = np.zeros((len(kept), H, D))
+    cnt = np.zeros((len(kept), H))
+    for h in range(H):
+        np.add.at(acc[:, h], match[h], v[h].astype(np.float64))
+        np.add.at(cnt[:, h], match[h], 1.0)
+    np.testing.assert_allclose(merged, acc / cnt[..., None], rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose((merged * cnt[..., None]).sum(axis=0), v.astype(np.float64).sum(axis=1), rtol=1e-12)
+    # nothing pruned: merging is plain compaction
+    full = np.arange(N, dtype=np.int32)
+    for mode in (oracle.MERGE_POSITION, oracle.MERGE_FEATURE):
+        m_all = oracle.merge_match(k, full, mode)
+        assert (m_all == np.arange(N)[None]).all()
+        np.testing.assert_array_equal(oracle.merge_rows(v, full, m_all), oracle.gather_rows(v, full).astype(np.float64))
+    # Position: nearest retained position, the lower one at equal distance, the same in every head
+    mp = oracle.merge_match(k, kept, oracle.MERGE_POSITION)
+    for m in range(N):
+        d = np.abs(kept.astype(np.int64) - m)
+        assert (mp[:, m] == int(np.argmin(d))).all()       # argmin takes the first (lowest) of equals
