@@ -218,6 +218,30 @@ int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strides ks, cons
                      size_t ws_bytes, void *cuda_stream);
 
 /*
+ * Compression with cache merging (Sec. 4.3, paragraph "Eviction or merging", Tab. "merge"):
+ * as prefixkv_compact, but a pruned vector is averaged into one retained vector instead of
+ * being dropped.  Per layer and head, each pruned key k^m is matched to the retained key k^n
+ * with the largest metric c^{mn}:
+ *   PKV_MERGE_POSITION   c^{mn} = -|m - n|
+ *   PKV_MERGE_FEATURE    c^{mn} = <k^m, k^n> / (|k^m| |k^n|)       (0 if a norm is 0)
+ * and the cached key / value of n becomes the plain average of its own vector and of the
+ * pruned vectors matched to it.  Where the paper is silent: the match is taken on the keys and
+ * applied to the values too; among equal metrics the retained vector at the lower position
+ * wins; averages are formed in fp32 and rounded once to the cache type.
+ *   kept    as for prefixkv_compact
+ *   match   [B,L,H,N] int32 out, may be NULL: for every position the index (into the
+ *           segment's ascending retained list) of the row it was merged into; a retained
+ *           position maps to its own row
+ * prompt_len <= 4096; not combined with decode-time pruning (evict_distance must be 0).
+ * Every prompt row of K and V is read once (not only the retained ones).
+ */
+enum { PKV_MERGE_POSITION = 1, PKV_MERGE_FEATURE = 2 };
+int prefixkv_compact_merge(const pkv_shape *shape, const void *k, pkv_strides ks, const void *v,
+                           pkv_strides vs, const int32_t *order, const int32_t *len,
+                           pkv_cache *cache, int32_t mode, int32_t *kept, int32_t *match,
+                           int32_t *dev_status, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * One decode step over the ragged cache (Sec. 3.1: the newest token attends over
  * the cached key/value vectors): for every segment of layers [layer_begin,
  * layer_end), append k_new / v_new as row len, then

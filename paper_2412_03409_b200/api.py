@@ -19,13 +19,14 @@ from . import build as _build
 (DEV_OK, DEV_BAD_SCORE, DEV_RANGE, DEV_BUDGET_TOO_SMALL, DEV_BAD_LENGTH, DEV_CAPACITY,
  DEV_TIMEOUT) = range(7)
 WS_SCORE, WS_SEARCH, WS_COMPACT, WS_DECODE = range(4)
+MERGE_POSITION, MERGE_FEATURE = 1, 2
 F32, BF16 = 0, 1
 
 EXPORTS = ["prefixkv_workspace_bytes", "prefixkv_last_cuda_error", "prefixkv_score",
            "prefixkv_search", "prefixkv_apply_lengths", "prefixkv_compact",
            "prefixkv_decode_attn", "prefixkv_gini", "prefixkv_rescale",
            "prefixkv_estimate_config", "prefixkv_decode_attn_static",
-           "prefixkv_selftest_bounded_wait", "prefixkv_decode_static_limit_bytes"]
+           "prefixkv_selftest_bounded_wait", "prefixkv_compact_merge", "prefixkv_decode_static_limit_bytes"]
 
 
 class Shape(ctypes.Structure):
@@ -77,6 +78,8 @@ def _load():
     lib.prefixkv_decode_attn_static.argtypes = [sp, ctypes.POINTER(CacheStruct), vp, vp, vp, vp,
                                                 i32, i32, vp, vp, vp]
     lib.prefixkv_selftest_bounded_wait.argtypes = [i32, vp, vp]
+    lib.prefixkv_compact_merge.argtypes = [sp, vp, Strides, vp, Strides, vp, vp, ctypes.POINTER(CacheStruct), i32,
+                                           vp, vp, vp, vp, sz, vp]
     for name in EXPORTS[2:-1]:
         getattr(lib, name).restype = ctypes.c_int
     lib.prefixkv_decode_static_limit_bytes.restype = ctypes.c_size_t
@@ -252,3 +255,10 @@ def prefixkv_estimate_config(shape, length, budget_rows, len_out, dev_status):
 def prefixkv_selftest_bounded_wait(which, dev_status):
     _check(_lib.prefixkv_selftest_bounded_wait(int(which), _ptr(dev_status), _stream()),
            "prefixkv_selftest_bounded_wait")
+
+
+def prefixkv_compact_merge(shape, k, v, order, length, cache: Cache, mode, dev_status, ws, kept=None, match=None):
+    p, n = _ws(ws)
+    _check(_lib.prefixkv_compact_merge(ctypes.byref(shape), _ptr(k), strides_of(k), _ptr(v), strides_of(v),
+                                       _ptr(order), _ptr(length), ctypes.byref(cache.c), int(mode), _ptr(kept),
+                                       _ptr(match), _ptr(dev_status), p, n, _stream()), "prefixkv_compact_merge")

@@ -139,6 +139,18 @@ gather_rows_kernel(const uint4 *__restrict__ k, const uint4 *__restrict__ v, pkv
     }
 }
 
+cudaError_t launch_compact_plan(const pkv_shape *shape, const int32_t *order, const int32_t *len, pkv_cache *cache,
+                                int32_t *kept, int32_t *dev_status, cudaStream_t stream)
+{
+    const int nseg = shape->batch * shape->layers;
+    const bool pruning = cache->evict_distance > 0;
+    return launch_dependent(compact_plan_kernel, dim3(nseg), dim3(1024), 0, stream, order, len, nseg, (int)shape->layers,
+                            (int)shape->prompt_len, cache->decode_cap, cache->total_cap_rows, cache->row_offset,
+                            cache->len, cache->cap, kept, dev_status, pruning ? cache->len0 : nullptr,
+                            pruning ? cache->gen : nullptr, pruning ? cache->slot_ring : nullptr,
+                            cache->evict_distance + 1);
+}
+
 }  // namespace pkv
 
 using namespace pkv;
@@ -171,11 +183,7 @@ extern "C" int prefixkv_compact(const pkv_shape *shape, const void *k, pkv_strid
     const bool pruning = cache->evict_distance > 0;
     if (pruning && (!cache->len0 || !cache->gen || !cache->slot_ring)) return PKV_ERR_INVALID_ARG;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    cudaError_t e = launch_dependent(compact_plan_kernel, dim3(nseg), dim3(1024), 0, stream, order, len, nseg, L, N,
-                                     cache->decode_cap, cache->total_cap_rows, cache->row_offset, cache->len,
-                                     cache->cap, kept, dev_status, pruning ? cache->len0 : nullptr,
-                                     pruning ? cache->gen : nullptr, pruning ? cache->slot_ring : nullptr,
-                                     cache->evict_distance + 1);
+    cudaError_t e = launch_compact_plan(shape, order, len, cache, kept, dev_status, stream);
     if (e != cudaSuccess) {
         set_cuda_error(e, "compact_plan_kernel");
         return PKV_ERR_CUDA;

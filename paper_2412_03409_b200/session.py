@@ -63,6 +63,10 @@ class Session:
         api.prefixkv_compact(self.shape, k, v, self.order, self.len, self.cache, self.status,
                              self.ws_compact, kept=self.kept)
 
+    def compact_merge(self, k, v, mode, match=None):
+        api.prefixkv_compact_merge(self.shape, k, v, self.order, self.len, self.cache, mode, self.status,
+                                   self.ws_compact, kept=self.kept, match=match)
+
     def compress(self, q, k, v, budget_rows, tol=1e-6, max_iters=64, slack_rows=0):
         self.score(q, k)
         self.search(budget_rows, tol, max_iters, slack_rows)

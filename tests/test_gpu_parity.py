@@ -679,3 +679,82 @@ def test_bounded_wait_reports_timeout(api, which):
     torch.cuda.synchronize()
     assert status.cpu().tolist() == [api.DEV_TIMEOUT, 0]
     assert int((torch.arange(8, device="cuda") + 1).sum()) == 36      # later work runs normally
+
+
+# --------------------------------------------------------------------------
+# cache merging (Sec. 4.3): pruned vectors averaged into the matched retained ones
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("name,kw", [
+    ("tiny", dict(N=90, H=3, L=2)),                        # fp32, D = 64
+    ("llava7b_b1", dict(L=2, H=4, N=333)),                 # bf16, D = 128, several 32-key tiles and a ragged one
+    ("llava7b_b16", dict(B=2, L=2, H=2, N=160, D=64)),
+])
+@pytest.mark.parametrize("mode", ["position", "feature"])
+def test_compact_with_merging_matches_oracle(api, name, kw, mode):
+    w = wl.scaled(wl.WORKLOADS[name], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 60) for b in range(w.B)])
+    s = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2, poison=True)
+    s.search(w.budget_rows(), scores=torch.from_numpy(scores).cuda())
+    code = api.MERGE_POSITION if mode == "position" else api.MERGE_FEATURE
+    match = torch.full((w.B, w.L, w.H, w.N), -7, dtype=torch.int32, device="cuda")
+    s.compact_merge(k, v, code, match=match)
+    torch.cuda.synchronize()
+    assert s.status.cpu().tolist() == [0] * w.B
+    tol = DECODE_TOL[w.dtype]
+    # merged rows are averages formed in fp32 and rounded once to the cache type: the error is the
+    # rounding of the result (half an ulp: 2^-9 relative for bf16, 2^-24 for fp32) plus the fp32
+    # summation of at most N terms; bound with a factor two of margin, relative with a floor of 1
+    rel = 2.0 ** -8 if w.dtype == torch.bfloat16 else 1e-5
+    for b in range(w.B):
+        for l in range(w.L):
+            n = int(s.len[b, l])
+            kept = oracle.retained_positions(s.order[b, l].cpu().numpy(), n)
+            np.testing.assert_array_equal(s.kept[b, l, :n].cpu().numpy(), kept)
+            got_match = match[b, l].cpu().numpy()
+            ref_match, gap = oracle.merge_match(to_np32(k[b, l]), kept, code, want_gap=True)
+            if mode == "position":
+                np.testing.assert_array_equal(got_match, ref_match)      # integer decisions: bit-exact
+            else:
+                # the argmax is decided in fp32 on the GPU and in fp64 by the oracle: they must agree
+                # wherever the best and second-best cosine differ by more than fp32 can blur; elsewhere
+                # the GPU's choice is one of the near-equal best and the rows are checked under it
+                differ = got_match != ref_match
+                assert not (differ & (gap > 1e-5)).any()
+                assert (got_match >= 0).all() and (got_match < n).all()
+            off = int(s.cache.row_offset[b * w.L + l])
+            for src, dst in ((k, s.cache.k), (v, s.cache.v)):
+                ref = oracle.merge_rows(to_np32(src[b, l]), kept, got_match)
+                got = to_np32(dst[off:off + n])
+                assert (np.abs(got - ref) <= rel * np.maximum(np.abs(ref), 1.0)).all()
+            # the head-room rows are untouched
+            assert torch.isnan(s.cache.k[off + n:off + n + 2].float()).all()
+    # decoding over the merged cache works like over any other
+    qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
+    out = to_np32(s.decode(qd, kn, vn))
+    b, l = w.B - 1, w.L - 1
+    off, n = int(s.cache.row_offset[b * w.L + l]), int(s.cache.len[b * w.L + l])
+    ref = oracle.decode_attn(to_np32(qd[b, l]), to_np32(s.cache.k[off:off + n]), to_np32(s.cache.v[off:off + n]),
+                             float(scale[l]))
+    assert np.abs(out[b, l] - ref).max() <= tol
+
+
+def test_merging_with_nothing_pruned_is_plain_compaction(api):
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=2, H=4, N=100)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scores = wl.synthetic_scores(w.L, w.N, seed=3)[None]
+    a = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, wl.layer_scale(w), decode_cap=1)
+    b = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, wl.layer_scale(w), decode_cap=1)
+    for s in (a, b):
+        s.search(w.L * w.N, scores=torch.from_numpy(scores).cuda())      # full budget: every row kept
+    a.compact(k, v)
+    b.compact_merge(k, v, api.MERGE_FEATURE)
+    torch.cuda.synchronize()
+    # (equal as values: an average of one vector is that vector, except that -0.0 comes out as +0.0)
+    for seg in range(w.L):
+        o = int(a.cache.row_offset[seg])
+        assert int(a.cache.len[seg]) == w.N
+        assert torch.equal(a.cache.k[o:o + w.N].float(), b.cache.k[o:o + w.N].float())
+        assert torch.equal(a.cache.v[o:o + w.N].float(), b.cache.v[o:o + w.N].float())
+    assert torch.equal(a.cache.len, b.cache.len) and torch.equal(a.cache.row_offset, b.cache.row_offset)
