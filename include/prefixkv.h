@@ -143,7 +143,8 @@ int prefixkv_search(const pkv_shape *shape, const float *scores, const int64_t *
  * Variant for a configuration fixed in advance (the offline estimate of
  * Sec. 3.3, last paragraph, or the uniform R_l = r of Sec. 3.2): ranks the rows
  * as above and takes the lengths from the caller.
- *   len_in   [L] (per_sample = 0) or [B,L] (per_sample = 1) int32, each in [1,N]
+ *   len_in   [L] (per_sample = 0) or [B,L] (per_sample = 1) int32, each in [1,N];
+ *            must not be the same buffer as `len`
  *   cum      may be NULL
  */
 int prefixkv_apply_lengths(const pkv_shape *shape, const float *scores, const int32_t *len_in,

@@ -493,10 +493,10 @@ int orc_apportion(const int64_t *weight, int L, int64_t budget, int N, int32_t *
 }
 
 /* ------------------------------------------------------------------------
- * Keeping the configuration while decoding (Sec. 3.1: "prune the vectors at a
- * fixed distance to the latest generated token and maintain the global prefix
- * configuration"; Fig. 2a: the cache "consistently maintains the derived
- * compression proportions").  The distance and the exact rule are left to the
+ * Keeping the configuration while decoding (Sec. 3.1: during generation the
+ * vectors at a fixed distance behind the newest token are pruned so that the
+ * layer-wise configuration is kept; Fig. 2a: the cache keeps the compression
+ * proportions found after prefilling).  The distance and the exact rule are left to the
  * cited work; reading used here, per layer:
  *   R_l = len0 / N is the layer's proportion.  When generated token g arrives
  *   (g = 0, 1, ...) the layer may hold floor(len0 * (N + g + 1) / N) rows.  If

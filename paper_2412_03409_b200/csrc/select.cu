@@ -35,7 +35,7 @@ __device__ __forceinline__ uint64_t add_check(uint64_t a, uint64_t b, bool &ovf)
 
 __global__ void __launch_bounds__(1024)
 sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t *__restrict__ order,
-                 uint64_t *__restrict__ cum, int32_t *dev_status)
+                 uint64_t *__restrict__ cum, int32_t *__restrict__ seg_flags)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint64_t *keys = reinterpret_cast<uint64_t *>(smem_raw);  // [P]
@@ -43,7 +43,6 @@ sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t 
     __shared__ int s_flags;
 
     const int seg = blockIdx.x;
-    const int b = seg / L;
     const int tid = threadIdx.x;
     const int nthr = blockDim.x;
     const float *src = scores + (size_t)seg * N;
@@ -146,8 +145,16 @@ sort_scan_kernel(const float *__restrict__ scores, int N, int P, int L, int32_t 
     if (bad) atomicOr(&s_flags, 1);
     if (range_bad || ovf) atomicOr(&s_flags, 2);
     __syncthreads();
-    if (tid == 0 && s_flags)
-        raise_status(dev_status, b, (s_flags & 1) ? PKV_DEV_BAD_SCORE : PKV_DEV_RANGE);
+    // What was found goes to the segment's slot of the length array (bit 0: a bad score, bit 1:
+    // the fixed-point range); the kernel that follows turns the flags of a sample's layers into
+    // its status word and then writes the lengths over them, so no separate clearing pass runs.
+    if (tid == 0) seg_flags[seg] = s_flags;
+}
+
+// Status of a sample from the flags the sort kernel left in its layers' length slots.
+__device__ __forceinline__ int status_from_flags(int flags)
+{
+    return (flags & 1) ? (int)PKV_DEV_BAD_SCORE : ((flags & 2) ? (int)PKV_DEV_RANGE : (int)PKV_DEV_OK);
 }
 
 // ---------------------------------------------------------------------------
@@ -194,8 +201,15 @@ search_kernel(const uint64_t *__restrict__ cum, const int64_t *__restrict__ budg
     const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
     const uint64_t *cb = cum + (size_t)b * L * N;
-    dependent_entry();  // the sort kernel's sums are complete
+    dependent_entry();  // the sort kernel's sums and flags are complete
     const int64_t budget = budget_rows[b];
+    {
+        int flags = 0;
+        for (int l = threadIdx.x; l < L; l += blockDim.x) flags |= len[(size_t)b * L + l];
+        // (the block-wide "or" is of predicates, so one per bit)
+        flags = (__syncthreads_or(flags & 1) ? 1 : 0) | (__syncthreads_or(flags & 2) ? 2 : 0);
+        if (threadIdx.x == 0) dev_status[b] = status_from_flags(flags);  // overwrites: this call's status starts here
+    }
 
     // What every midpoint needs of a layer's row and never changes: its total and this lane's
     // first-round probe.  Kept in registers for the first kHoist layers of the warp.
@@ -289,27 +303,33 @@ search_kernel(const uint64_t *__restrict__ cum, const int64_t *__restrict__ budg
     }
 }
 
-__global__ void clear_status_kernel(int32_t *dev_status, int B)
+// One CTA per sample: the caller's lengths, checked, and the sample's status word.
+__global__ void __launch_bounds__(256)
+take_lengths_kernel(const int32_t *__restrict__ len_in, int per_sample, int L, int N,
+                    int32_t *__restrict__ len, int32_t *dev_status)
 {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < B) dev_status[i] = PKV_DEV_OK;
-}
-
-__global__ void take_lengths_kernel(const int32_t *__restrict__ len_in, int per_sample, int B, int L,
-                                    int N, int32_t *__restrict__ len, int32_t *dev_status)
-{
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= B * L) return;
-    int v = per_sample ? len_in[i] : len_in[i % L];
-    if (v < 1 || v > N) {
-        raise_status(dev_status, i / L, PKV_DEV_BAD_LENGTH);
-        v = v < 1 ? 1 : N;
+    const int b = blockIdx.x;
+    dependent_entry();  // the sort kernel's flags are complete
+    int flags = 0, bad = 0;
+    for (int l = threadIdx.x; l < L; l += blockDim.x) {
+        flags |= len[(size_t)b * L + l];
+        int v = per_sample ? len_in[(size_t)b * L + l] : len_in[l];
+        if (v < 1 || v > N) {
+            bad = 1;
+            v = v < 1 ? 1 : N;
+        }
+        len[(size_t)b * L + l] = v;
     }
-    len[i] = v;
+    flags = (__syncthreads_or(flags & 1) ? 1 : 0) | (__syncthreads_or(flags & 2) ? 2 : 0);  // predicates: one per bit
+    bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
+        const int st = status_from_flags(flags);
+        dev_status[b] = st != PKV_DEV_OK ? st : (bad ? (int)PKV_DEV_BAD_LENGTH : (int)PKV_DEV_OK);
+    }
 }
 
 static int launch_sort(const pkv_shape *s, const float *scores, int32_t *order, uint64_t *cum,
-                       int32_t *dev_status, cudaStream_t st)
+                       int32_t *seg_flags, cudaStream_t st)
 {
     int N = s->prompt_len;
     int P = 32;
@@ -322,7 +342,7 @@ static int launch_sort(const pkv_shape *s, const float *scores, int32_t *order, 
         if (rc != PKV_OK) return rc;
     }
     cudaError_t e = launch_dependent(sort_scan_kernel, dim3(s->batch * s->layers), dim3(nthr), smem, st, scores, N, P,
-                                     (int)s->layers, order, cum, dev_status);
+                                     (int)s->layers, order, cum, seg_flags);
     if (e != cudaSuccess) {
         set_cuda_error(e, "sort_scan_kernel");
         return PKV_ERR_CUDA;
@@ -348,8 +368,7 @@ extern "C" int prefixkv_search(const pkv_shape *shape, const float *scores,
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int B = shape->batch, L = shape->layers, N = shape->prompt_len;
     if ((size_t)2 * L * sizeof(int) > 40 * 1024) return PKV_ERR_UNSUPPORTED;
-    clear_status_kernel<<<(B + 255) / 256, 256, 0, st>>>(dev_status, B);
-    int rc = launch_sort(shape, scores, order, cum, dev_status, st);
+    int rc = launch_sort(shape, scores, order, cum, len, st);
     if (rc != PKV_OK) return rc;
     cudaError_t e = launch_dependent(search_kernel, dim3(B), dim3(1024), 2 * L * sizeof(int), st,
                                      (const uint64_t *)cum, budget_rows, L, N, tol, (int)max_iters, slack_rows, slack_over_rows, len,
@@ -372,10 +391,14 @@ extern "C" int prefixkv_apply_lengths(const pkv_shape *shape, const float *score
     if (!shape_supported(shape)) return PKV_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int B = shape->batch, L = shape->layers, N = shape->prompt_len;
-    clear_status_kernel<<<(B + 255) / 256, 256, 0, st>>>(dev_status, B);
-    int rc = launch_sort(shape, scores, order, cum, dev_status, st);
+    if (len_in == len) return PKV_ERR_INVALID_ARG;  // (the output slots carry the sort's flags in between)
+    int rc = launch_sort(shape, scores, order, cum, len, st);
     if (rc != PKV_OK) return rc;
-    take_lengths_kernel<<<(B * L + 255) / 256, 256, 0, st>>>(len_in, per_sample, B, L, N, len,
-                                                             dev_status);
-    return check_launch("take_lengths_kernel");
+    cudaError_t e = launch_dependent(take_lengths_kernel, dim3(B), dim3(256), 0, st, len_in, (int)per_sample, L, N, len,
+                                     dev_status);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "take_lengths_kernel");
+        return PKV_ERR_CUDA;
+    }
+    return PKV_OK;
 }
