@@ -478,9 +478,9 @@ def run_ours(args):
 
 
 def LAUNCHES_PER_STEP(w):
-    # score: lse + column sums + head mean; search: status clear + sort/scan + bisection;
+    # score: lse + column sums + head mean; search: sort/scan + bisection;
     # compact: plan + gather; decode: stream + merge per token
-    return 3 + 3 + 2 + 2 * w.T
+    return 3 + 2 + 2 + 2 * w.T
 
 
 def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):
