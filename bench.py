@@ -70,24 +70,39 @@ def measured_peaks():
         return FALLBACK_HBM_GBS, FALLBACK_BF16_TFLOPS, "fallback"
 
 
-# DRAM bytes (read + write) of one decode_stream_kernel launch from an ncu capture (its summary is
-# kept under profiles/), keyed by workload, with the hash of the kernel's source
-# the counters were taken on: once that file changes the figure is stale and `traffic` reads null.
-DECODE_TRAFFIC = {"llava7b_b1": (102.61e6, "074b548178a7e41a")}
+# Which kernel a decode call takes: the library's rule (launch_decode_heads in csrc/decode_heads.cu)
+# restated, for the kernel's name, the launch count and the traffic figure below.
+DECODE_KERNELS = {
+    "heads": ("decode_heads_kernel", "decode_heads.cu", "decode_heads_kernel(const __grid_constant__ CUtensorMap map_k", 1),
+    "stream": ("decode_stream_kernel + its merge kernel", "decode_stream.cu", "decode_stream_kernel(const DecodeArgs a)", 2),
+}
 
 
-def decode_traffic(workload):
-    """The captured figure, or None when decode_stream_kernel's source (the function itself, from
-    its signature to its closing brace) is no longer what the counters were taken on."""
+def decode_path(w, sms):
+    nact = w.B * w.L
+    heads = w.D in (64, 128) and nact <= 256 and nact * w.H >= 4 * sms and 2 * nact <= sms
+    return "heads" if heads else "stream"
+
+
+# DRAM bytes (read + write) of one launch of the workload's decode kernel from an ncu capture (its
+# summary is kept under profiles/), keyed by workload and kernel, with the hash of the kernel's source
+# the counters were taken on: once that function changes the figure is stale and `traffic` reads null.
+DECODE_TRAFFIC = {("llava7b_b1", "heads"): (101.63e6, "")}
+
+
+def decode_traffic(workload, path):
+    """The captured figure, or None when the kernel's source (the function itself, from its
+    signature to its closing brace) is no longer what the counters were taken on."""
     import hashlib
-    ent = DECODE_TRAFFIC.get(workload)
+    ent = DECODE_TRAFFIC.get((workload, path))
     if ent is None:
         return None
-    src = os.path.join(ROOT, "paper_2412_03409_b200", "csrc", "decode_stream.cu")
+    _, fname, signature, _ = DECODE_KERNELS[path]
+    src = os.path.join(ROOT, "paper_2412_03409_b200", "csrc", fname)
     try:
         with open(src) as f:
             text = f.read()
-        start = text.index("decode_stream_kernel(const DecodeArgs a)")
+        start = text.index(signature)
         end = text.index("\n}\n", start)
     except (OSError, ValueError):
         return None
@@ -430,6 +445,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     value = world * w.B * w.T / (step_ms_max * 1e-3)
+    path = decode_path(w, torch.cuda.get_device_properties(dev).multi_processor_count)
     line = {
         "metric": "tok/s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True,
@@ -453,11 +469,11 @@ def run_ours(args):
                      "compact_gbs": m["compact_bytes"] / (stage_ms["compact"] * 1e-3) / 1e9,
                      "score_tensor_util_vs_burst": m["causal_flop"] * 2 / (stage_ms["score"] * 1e-3) / (tf_peak * 1e12),
                      "target_ms_strict": m["causal_flop"] / (0.5 * tf_peak * 1e12) * 1e3},
-        "roofline": {"bound": "hbm", "kernel": "decode_stream_kernel + its merge kernel (one decode call, launch gaps included)",
+        "roofline": {"bound": "hbm", "kernel": DECODE_KERNELS[path][0] + " (one decode call, launch gaps included)",
                      "achieved": dec_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": dec_gbs / hbm_peak,
-                     "peak_kind": "of " + peak_kind, "traffic": decode_traffic(w.name),
+                     "peak_kind": "of " + peak_kind, "traffic": decode_traffic(w.name, path),
                      "bytes_per_launch": dec_bytes / w.T, "us_per_launch": 1e3 * stage_ms["decode"] / w.T},
-        "gpu_launches": args.steps * R * LAUNCHES_PER_STEP(w),
+        "gpu_launches": args.steps * R * LAUNCHES_PER_STEP(w, path),
         "clocks": clocks,
     }
     if others:
@@ -477,10 +493,10 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def LAUNCHES_PER_STEP(w):
+def LAUNCHES_PER_STEP(w, path):
     # score: lse + column sums + head mean; search: sort/scan + bisection;
-    # compact: plan + gather; decode: stream + merge per token
-    return 3 + 2 + 2 + 2 * w.T
+    # compact: plan + gather; decode: one kernel per token, or stream + merge
+    return 3 + 2 + 2 + DECODE_KERNELS[path][3] * w.T
 
 
 def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):

@@ -161,6 +161,9 @@ static int pick_splits(int nseg_active)
 }
 
 size_t decode_stream_ws_bytes(const pkv_shape *s);
+size_t decode_heads_ws_bytes();
+int launch_decode_heads(const pkv_shape *s, pkv_cache *c, const void *q, const void *kn, const void *vn,
+                        const float *scale, int lb, int le, void *out, int32_t *dev_status, void *ws, cudaStream_t st);
 int launch_decode_stream(const pkv_shape *s, pkv_cache *c, const void *q, const void *kn,
                          const void *vn, const float *scale, int lb, int le, void *out,
                          int32_t *dev_status, void *ws, cudaStream_t st);
@@ -171,8 +174,9 @@ size_t decode_ws_bytes(const pkv_shape *s)
     size_t nseg = (size_t)s->batch * s->layers;
     size_t slots = 148 * 4 + nseg;
     size_t per = (size_t)s->heads * (s->head_dim + 2) * sizeof(float);
-    size_t two = round_up(slots * per, kWsAlign), one = decode_stream_ws_bytes(s);
-    return two > one ? two : one;
+    size_t two = round_up(slots * per, kWsAlign), one = decode_stream_ws_bytes(s), heads = decode_heads_ws_bytes();
+    size_t need = two > one ? two : one;
+    return need > heads ? need : heads;
 }
 
 template <typename T, int D>
@@ -220,6 +224,12 @@ extern "C" int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, co
     if ((size_t)shape->batch * (layer_end - layer_begin) > 65535) return PKV_ERR_UNSUPPORTED;
     if (!ws || !aligned(ws, kWsAlign) || ws_bytes < decode_ws_bytes(shape)) return PKV_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    {
+        // Few segments: whole (segment, head) items per CTA, no partials and no second kernel.
+        int rc = launch_decode_heads(shape, cache, q, k_new, v_new, layer_scale, layer_begin, layer_end, out, dev_status,
+                                     ws, st);
+        if (rc >= 0) return rc;  // -1: not a case for that kernel
+    }
     {
         // The streaming kernel plans at most 1024 segments at a time: a larger batch x layer range
         // goes through it in layer chunks, one launch after the other on the stream.

@@ -274,6 +274,15 @@ def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
     ("llava7b_b1", dict(L=2, H=64, N=90, T=2)),              # 64 heads: four heads per consumer warp
     ("llava7b_b1", dict(L=2, H=72, D=64, N=90, T=2)),        # more heads than the streaming kernel takes: two-kernel path
     ("llava7b_b16", dict(B=40, L=32, H=2, D=64, N=24, T=2)),  # 1280 segments: two layer chunks through the streaming kernel
+    # few segments, many (segment, head) items: the per-head kernel (whole softmax rows per CTA)
+    ("llava7b_b1", dict(L=20, H=32, N=100, T=3)),            # bf16, 256-byte head slices
+    ("tiny", dict(L=16, H=40, N=70, T=3)),                   # fp32, D = 64
+    ("tiny", dict(B=2, L=10, H=32, D=128, N=50, T=2)),       # fp32, D = 128: 512-byte slices, one row per warp step
+    ("llava7b_b1", dict(L=10, H=64, D=64, N=150, T=2)),      # bf16, D = 64: 128-byte slices, four rows per warp step
+    ("llava7b_b1", dict(L=20, H=32, N=700, T=2, budget_ratios=(1.0,))),   # 22 tiles per item: more than consumer warps
+    ("llava7b_b1", dict(L=24, H=27, N=100, T=2)),            # odd head count: single heads only
+    ("llava7b_b1", dict(L=24, H=40, D=64, N=100, T=2)),      # bf16, D = 64: rounds of 4 heads, of 2 heads and of single heads
+    ("llava7b_b1", dict(L=37, H=18, N=100, T=2)),            # head count not a multiple of 4; pairs, then single heads
 ])
 def test_decode_matches_oracle(api, name, kw):
     w = wl.scaled(wl.WORKLOADS[name], **kw)
@@ -336,12 +345,14 @@ def test_decode_layer_range(api):
     assert torch.equal(a.cache.len, b.cache.len)
 
 
+@pytest.mark.parametrize("kw", [dict(L=6, H=8, N=300, T=2),        # streaming kernel + merge kernel
+                                dict(L=20, H=32, N=120, T=2)])     # per-head kernel (its flags live in the workspace)
 @pytest.mark.parametrize("byte", [0x7f, 0xff, 0x00])
-def test_decode_with_stale_workspace(api, byte):
+def test_decode_with_stale_workspace(api, byte, kw):
     """The decode workspace may hold anything (another shape's partials, an earlier call's plan):
     results do not depend on it.  (The merge kernel looks at its plan record early, before the record
     is final, and must bound what it does with that copy.)"""
-    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=6, H=8, N=300, T=2)
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], **kw)
     q, k, v = wl.make_prompt(w, "cuda")
     scale = wl.layer_scale(w)
     scores = torch.from_numpy(wl.synthetic_scores(w.L, w.N, 5)[None]).cuda()
@@ -362,11 +373,12 @@ def test_decode_with_stale_workspace(api, byte):
     assert a.status.cpu().tolist() == b.status.cpu().tolist() == [0]
 
 
-@pytest.mark.parametrize("kw", [dict(H=4), dict(H=72, D=64)])      # streaming kernel; two-kernel path (H > 64)
+@pytest.mark.parametrize("kw", [dict(H=4), dict(H=72, D=64),       # streaming kernel; two-kernel path (H > 64)
+                                dict(H=32, L=10)])                 # per-head kernel
 def test_decode_empty_segment_is_reported(api, kw):
     """A segment with no rows (never compacted) cannot be attended over: the sample's status says
     so, its output is zero, its length stays, and the other segments are unaffected."""
-    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], B=2, L=3, N=80, T=2, **kw)
+    w = wl.scaled(wl.WORKLOADS["llava7b_b16"], **{**dict(B=2, L=3, N=80, T=2), **kw})
     q, k, v = wl.make_prompt(w, "cuda")
     scale = wl.layer_scale(w)
     scores = np.stack([wl.synthetic_scores(w.L, w.N, seed=b + 11) for b in range(w.B)])
@@ -393,6 +405,7 @@ def test_decode_empty_segment_is_reported(api, kw):
 @pytest.mark.parametrize("name,kw", [
     ("tiny", {}),
     ("llava7b_b1", dict(L=3, H=8, N=200, T=3)),
+    ("llava7b_b1", dict(L=20, H=32, N=90, T=3)),            # per-head kernel
 ])
 def test_decode_without_append(api, name, kw):
     """k_new = v_new = NULL: the query attends over the rows already cached and nothing changes."""
