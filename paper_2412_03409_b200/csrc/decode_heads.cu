@@ -24,7 +24,9 @@
 // (half the rows each) 22.4; an item's last, partial tile fetched in quarter-tile boxes 22.6 with
 // five producers, 27.3 with one; neighbouring heads fetched side by side in boxes twice as wide
 // and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7;
-// launched without the programmatic dependency 24.0.
+// launched without the programmatic dependency 24.0; an item's partial last tile read by its warp
+// straight from global memory (no bytes past the length) 27.0: plain loads queue behind the bulk
+// copies in flight, and the last item's two round trips end the kernel.
 #include <cuda.h>
 
 #include <atomic>
