@@ -42,6 +42,9 @@ constexpr int kHWarps = 10;        // consumer warps; warp kHWarps is the produc
 constexpr int kHStages = kHWarps;  // tiles in flight per CTA: warp w owns stage w, so that every stage has one
                                    // consumer that sees each of its phases in turn (with more warps than stages a
                                    // warp would skip phases of a stage and a parity wait could pass a cycle early)
+constexpr int kHPrefetch = 4;      // tiles of each of the CTA's first kHPrefetchItems items asked into L2 while the
+constexpr int kHPrefetchItems = 1;  // kernel before this one drains, one lane per tile (more measured no better)
+static_assert(kHPrefetch * kHPrefetchItems <= 32, "one lane per prefetched tile");
 constexpr int kHSlots = 4;         // items whose partial results may be waiting for their last tile
 constexpr int kHMaxAct = 256;      // segments planned per call
 constexpr int kHMaxGrid = 256;
@@ -126,6 +129,13 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, u
 __device__ __forceinline__ void prefetch_map(const CUtensorMap *map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+// Ask for a box to be brought into L2 (nothing is waited for, nothing lands in shared memory).
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap *map, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(map)),
+                 "r"(x), "r"(y)
+                 : "memory");
 }
 __device__ __forceinline__ void hbulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
@@ -216,7 +226,26 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // Launched as a programmatic dependent of whatever precedes it in the stream: the set-up above
-    // overlapped that kernel's tail; its writes (lengths, cache rows) are visible from here.
+    // overlaps that kernel's tail, and so does this: the first tiles of the CTA's first item are
+    // asked into L2 (a prefetch, so nothing is read into the SM before the wait; the rows' place
+    // comes from row_offset and cap, which decode calls do not write -- were they still being
+    // written by a compaction, the boxes asked for would be other, harmless ones: a tensor-map
+    // copy cannot leave the cache).  When the wait returns, the memory system has had the otherwise
+    // idle tail of the earlier kernel to fetch them.
+    if (warp == kHWarps && lane < kHPrefetch * kHPrefetchItems) {
+        const int it = (int)blockIdx.x + (lane / kHPrefetch) * (int)gridDim.x, t = lane % kHPrefetch;
+        if (it < a.nact * H) {
+            const int si = it / H, h = it - si * H;
+            const int seg = (si / a.nl) * a.L + a.layer_begin + si % a.nl;
+            const long long off = a.row_offset[seg];
+            const int cp = a.cap[seg];
+            if (off >= 0 && off + cp <= a.total_cap_rows && t * TILE_ROWS < cp) {
+                tma_prefetch_2d(&map_k, h * D, (int)off + t * TILE_ROWS);
+                tma_prefetch_2d(&map_v, h * D, (int)off + t * TILE_ROWS);
+            }
+        }
+    }
+    // Its writes (lengths, cache rows) are visible from here.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
