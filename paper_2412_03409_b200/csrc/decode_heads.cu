@@ -20,7 +20,8 @@
 // new lengths, so no CTA can read a length of the next step.  Every wait is bounded.
 //
 // Measured on the 32-layer, 32-head, 128-rows-per-layer case (22.3 us per call with this design),
-// each alone: one producer thread 24.1 us, five 22.9, ten 23.1; two consumer warps per tile
+// each alone: one producer thread 24.1 us, five 22.9, ten 23.1; eight stages 22.4, twelve 21.9 (with
+// the prefetch below, against 21.95 for ten); two consumer warps per tile
 // (half the rows each) 22.4; an item's last, partial tile fetched in quarter-tile boxes 22.6 with
 // five producers, 27.3 with one; neighbouring heads fetched side by side in boxes twice as wide
 // and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7;

@@ -326,11 +326,15 @@ def test_decode_full_budget_is_dense_attention(api):
         assert (out[0, l] - ref).abs().max() <= DECODE_TOL[w.dtype]
 
 
-def test_decode_layer_range(api):
-    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], L=4, H=4, N=80, T=2)
+@pytest.mark.parametrize("kw,step", [
+    (dict(L=4, H=4, N=80, T=2), 1),                 # a model calls one layer at a time (streaming kernel)
+    (dict(B=2, L=20, H=32, N=70, T=2), 10),         # two samples, ten layers per call: the per-head kernel on a sub-range
+])
+def test_decode_layer_range(api, kw, step):
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], **kw)
     q, k, v = wl.make_prompt(w, "cuda")
     scale = wl.layer_scale(w)
-    scores = torch.from_numpy(wl.synthetic_scores(w.L, w.N, 4)[None]).cuda()
+    scores = torch.from_numpy(np.stack([wl.synthetic_scores(w.L, w.N, 4 + b) for b in range(w.B)])).cuda()
     a = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
     b = _session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=2)
     for s in (a, b):
@@ -339,8 +343,8 @@ def test_decode_layer_range(api):
     qd, kn, vn = wl.make_decode_inputs(w, 0, "cuda")
     full = a.decode(qd, kn, vn).float().clone()
     b.out.zero_()
-    for l in range(w.L):                      # a model calls one layer at a time
-        b.decode(qd, kn, vn, layer_begin=l, layer_end=l + 1)
+    for l in range(0, w.L, step):
+        b.decode(qd, kn, vn, layer_begin=l, layer_end=l + step)
     assert (full - b.out.float()).abs().max() <= DECODE_TOL[w.dtype]
     assert torch.equal(a.cache.len, b.cache.len)
 
