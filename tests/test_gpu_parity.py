@@ -280,9 +280,10 @@ def _decode_reference(w, s, k, v, ref_sel, steps, layer_scale):
     ("tiny", dict(B=2, L=10, H=32, D=128, N=50, T=2)),       # fp32, D = 128: 512-byte slices, one row per warp step
     ("llava7b_b1", dict(L=10, H=64, D=64, N=150, T=2)),      # bf16, D = 64: 128-byte slices, four rows per warp step
     ("llava7b_b1", dict(L=20, H=32, N=700, T=2, budget_ratios=(1.0,))),   # 22 tiles per item: more than consumer warps
-    ("llava7b_b1", dict(L=24, H=27, N=100, T=2)),            # odd head count: single heads only
-    ("llava7b_b1", dict(L=24, H=40, D=64, N=100, T=2)),      # bf16, D = 64: rounds of 4 heads, of 2 heads and of single heads
-    ("llava7b_b1", dict(L=37, H=18, N=100, T=2)),            # head count not a multiple of 4; pairs, then single heads
+    ("llava7b_b1", dict(L=24, H=27, N=100, T=2)),            # odd head count
+    ("llava7b_b1", dict(L=24, H=40, D=64, N=100, T=2)),      # bf16, D = 64, 40 heads
+    ("llava7b_b1", dict(L=37, H=18, N=100, T=2)),            # 666 items over 148 CTAs: four or five each
+    ("llava7b_b1", dict(B=4, L=32, H=8, N=60, T=2)),         # 128 segments (several samples) on the per-head kernel
 ])
 def test_decode_matches_oracle(api, name, kw):
     w = wl.scaled(wl.WORKLOADS[name], **kw)
