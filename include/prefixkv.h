@@ -259,6 +259,9 @@ int prefixkv_compact_merge(const pkv_shape *shape, const void *k, pkv_strides ks
  * g - d is still cached, the new row takes that token's slot and len stays; otherwise it is
  * appended.  Prompt rows are never dropped.  Calls on one cache, or sharing one workspace, must not overlap on
  * the GPU.
+ * The call only enqueues kernels on cuda_stream, so it may be captured into a CUDA graph and
+ * replayed once per token (same pointers, new contents); make one call on the device outside
+ * any capture first, which sets the kernels up.
  */
 int prefixkv_decode_attn(const pkv_shape *shape, pkv_cache *cache, const void *q,
                          const void *k_new, const void *v_new, const float *layer_scale,

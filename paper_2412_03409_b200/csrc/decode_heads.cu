@@ -546,6 +546,9 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             }
         }
         if (__syncthreads_and(all_in)) {
+            // (flags go back to zero, which no token is: a call replayed from a CUDA graph comes
+            // with the same token and must not find the flags of its previous run)
+            if (tid < (int)gridDim.x) a.flags[tid] = 0ull;
             for (int si = tid; si < a.nact; si += blockDim.x)
                 if (s_len[si] >= 0) a.len[(si / a.nl) * a.L + a.layer_begin + si % a.nl] = s_len[si] + 1;
         } else if (tid == 0) {

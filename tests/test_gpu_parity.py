@@ -350,6 +350,37 @@ def test_decode_layer_range(api, kw, step):
     assert torch.equal(a.cache.len, b.cache.len)
 
 
+@pytest.mark.parametrize("kw", [dict(L=6, H=8, N=300, T=5),        # streaming kernel + merge kernel
+                                dict(L=20, H=32, N=100, T=5)])     # per-head kernel
+def test_decode_replayed_from_a_cuda_graph(api, kw):
+    """One decode call captured in a CUDA graph and replayed token after token gives, bit for bit,
+    what separate calls give: nothing a call leaves behind (lengths, workspace flags) may depend
+    on its being launched afresh."""
+    w = wl.scaled(wl.WORKLOADS["llava7b_b1"], **kw)
+    q, k, v = wl.make_prompt(w, "cuda")
+    scale = wl.layer_scale(w)
+    scores = torch.from_numpy(wl.synthetic_scores(w.L, w.N, 9)[None]).cuda()
+    a, b, warm = (_session(w.B, w.L, w.H, w.D, w.N, w.dtype, scale, decode_cap=w.T) for _ in range(3))
+    for s in (a, b, warm):
+        s.search(w.budget_rows(), scores=scores)
+        s.compact(k, v)
+    sq, sk, sv = (t.clone() for t in wl.make_decode_inputs(w, 0, "cuda"))
+    warm.decode(sq, sk, sv)                   # one-off set-up of the kernels happens outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        b.decode(sq, sk, sv)
+    for t in range(w.T):
+        qd, kn, vn = wl.make_decode_inputs(w, t, "cuda")
+        sq.copy_(qd); sk.copy_(kn); sv.copy_(vn)
+        graph.replay()
+        ref = a.decode(qd, kn, vn)
+        torch.cuda.synchronize()
+        assert torch.equal(b.out, ref), t
+        assert torch.equal(a.cache.len, b.cache.len), t
+    assert int(b.status.max()) == 0
+
+
 @pytest.mark.parametrize("kw", [dict(L=6, H=8, N=300, T=2),        # streaming kernel + merge kernel
                                 dict(L=20, H=32, N=120, T=2)])     # per-head kernel (its flags live in the workspace)
 @pytest.mark.parametrize("byte", [0x7f, 0xff, 0x00])
