@@ -421,7 +421,7 @@ def run_ours(args):
 
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, max(2, min(args.steps, 5)))
+        e2e = run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, max(2, min(args.steps, 20)))
         e2e["ms"] = sharding.max_over_ranks(e2e["ms"], dev)
     del m["reps"], s, q, k, v
     torch.cuda.empty_cache()
@@ -484,8 +484,8 @@ def run_ours(args):
         line["e2e"] = {"value": world * w.B * w.T / (e2e["ms"] * 1e-3), "unit": "tok/s",
                        "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                        "note": "host pinned Q,K,V and per-token q,k,v copied in, outputs copied out and "
-                               "synchronised per token; the next prompt uploads on a copy stream while "
-                               "this one decodes; wall clock over the steps, no L2 flush"}
+                               "synchronised per token; the next prompt uploads on a copy stream, one piece "
+                               "per token, while this one decodes; wall clock over the steps, no L2 flush"}
     if world == 1 and not args.no_cpu_baseline:
         v_cpu, desc, spent = time_oracle_sample(w, score_layers=min(w.L, 16), decode_steps=(0, 1, 2, 3))
         line["cpu_baseline"] = {"value": v_cpu, "unit": "tok/s", "cores": 1, "kind": "oracle",
@@ -505,8 +505,8 @@ def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):
     """Same path with host buffers: every step's prompt tensors start in pinned host memory and every
     token's q, k, v are copied in and its output copied out, with a host synchronisation per token
     (the result is needed before the next token).  The way a serving loop would run it: the next
-    prompt's upload goes through a copy stream into a second set of device buffers while the
-    current prompt decodes; a token's three inputs travel as one copy."""
+    prompt's upload goes through a copy stream into a second set of device buffers, piece by piece
+    between the tokens of the current prompt; a token's three inputs travel as one copy."""
     hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
     hpool = [torch.stack([x.cpu() for x in p]).pin_memory() for p in pool]      # [3, B, L, H, D] per token
     dbuf = [tuple(torch.empty_like(t) for t in (q, k, v)) for _ in range(2)]
@@ -519,20 +519,46 @@ def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):
     ready = [torch.cuda.Event() for _ in range(2)]
     free = [torch.cuda.Event() for _ in range(2)]
 
-    def upload(i):
+    # The upload of the next prompt is cut into one piece per token of the current prompt (a run of
+    # (layer, head) slices of Q, K or V, 3.75 MB here), handed to the copy stream right behind the
+    # token's own inputs: all host-to-device copies go through one engine in the order they were
+    # submitted, so a token's small copy queued behind a 160 MB one waited milliseconds for it,
+    # while a piece of this size crosses the link in the time the token takes to compute, come
+    # back and be followed by the next.
+    def pieces(i):
+        flat = [(d_.flatten(0, 2), h_.flatten(0, 2)) for d_, h_ in zip(dbuf[i % 2], (hq, hk, hv))]  # [B*L*H, N, D] each
+        rows = flat[0][0].shape[0]
+        per = -(-len(flat) * rows // w.T)
+        out = []
+        for t in range(w.T):
+            todo = []
+            for r in range(t * per, min((t + 1) * per, len(flat) * rows)):
+                todo.append((r // rows, r % rows))
+            runs = []
+            for which, r in todo:                       # consecutive rows of one tensor travel as one copy
+                if runs and runs[-1][0] == which and runs[-1][2] == r:
+                    runs[-1][2] = r + 1
+                else:
+                    runs.append([which, r, r + 1])
+            out.append([(flat[which][0][a:b], flat[which][1][a:b]) for which, a, b in runs])
+        return out
+
+    def send(todo):
         with torch.cuda.stream(copy):
-            copy.wait_event(free[i % 2])            # the buffers' previous prompt has been compacted
-            for d_, h_ in zip(dbuf[i % 2], (hq, hk, hv)):
+            for d_, h_ in todo:
                 d_.copy_(h_, non_blocking=True)
-            ready[i % 2].record(copy)
 
     def run(n):
         for e in free:
             e.record(main)
-        upload(0)
+        copy.wait_event(free[0])
+        for todo in pieces(0):
+            send(todo)
+        ready[0].record(copy)
         for i in range(n):
-            if i + 1 < n:
-                upload(i + 1)
+            nxt = pieces(i + 1) if i + 1 < n else []
+            if nxt:
+                copy.wait_event(free[(i + 1) % 2])  # the buffers' previous prompt has been compacted
             dq, dk, dv = dbuf[i % 2]
             main.wait_event(ready[i % 2])
             s.score(dq, dk)
@@ -541,9 +567,14 @@ def run_e2e(torch, api, w, s, q, k, v, pool, budget, dev, steps):
             free[i % 2].record(main)
             for t in range(w.T):
                 dtok.copy_(hpool[t % len(hpool)], non_blocking=True)
+                # (right behind the token's inputs, so that they cross the link while the token is computed)
+                if nxt:
+                    send(nxt[t])
                 s.decode(dtok[0], dtok[1], dtok[2])
                 hout.copy_(s.out, non_blocking=True)
                 main.synchronize()                # the token's result is needed on the host
+            if nxt:
+                ready[(i + 1) % 2].record(copy)
 
     run(1)
     torch.cuda.synchronize()
