@@ -7,8 +7,9 @@
 // A head's slice of a token-major cache row is D elements out of H * D, so an item's K (or V)
 // is a strided 2-D box: producer threads fetch 8 KiB tiles of it (rows x one head) with
 // cp.async.bulk.tensor through a rank-2 tensor map over [rows][H * D] (this GPU's own memory, no
-// multicast), together with the head's q and, for the item's last tile, the head's slice of the
-// new k / v row.  Issuing one of these copies holds its thread for some hundred cycles whatever
+// multicast; an item's last tile with the lowest of four box heights that holds its rows, so that
+// little is read past the segment's length), together with the head's q and, for the item's last
+// tile, the head's slice of the new k / v row.  Issuing one of these copies holds its thread for some hundred cycles whatever
 // its size, so two producer threads (one per warp) share the tiles: tile g is issued by producer
 // g mod 2.  Ten consumer warps take the tiles of the CTA's stream in turn (tile g goes to warp
 // g mod 10, through stage g mod 10), keep a running fp32 softmax state for the item they are in,
@@ -25,13 +26,15 @@
 // (half the rows each) 22.4; an item's last, partial tile fetched in quarter-tile boxes 22.6 with
 // five producers, 27.3 with one; neighbouring heads fetched side by side in boxes twice as wide
 // and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7;
-// launched without the programmatic dependency 24.0; an item's partial last tile read by its warp
+// launched without the programmatic dependency 24.0 (all these with whole boxes for every tile;
+// choosing the last tile's box among four heights then took 21.95 to 21.15); an item's partial last tile read by its warp
 // straight from global memory (no bytes past the length) 27.0: plain loads queue behind the bulk
 // copies in flight, and the last item's two round trips end the kernel.
 #include <cuda.h>
 
 #include <atomic>
 #include <chrono>
+#include <mutex>
 
 #include "common.cuh"
 
@@ -43,6 +46,7 @@ constexpr int kHWarps = 10;        // consumer warps; warp kHWarps is the produc
 constexpr int kHStages = kHWarps;  // tiles in flight per CTA: warp w owns stage w, so that every stage has one
                                    // consumer that sees each of its phases in turn (with more warps than stages a
                                    // warp would skip phases of a stage and a parity wait could pass a cycle early)
+constexpr int kHHeights = 4;       // box heights to choose from for an item's last tile (eight measured no better)
 constexpr int kHPrefetch = 4;      // tiles of each of the CTA's first kHPrefetchItems items asked into L2 while the
 constexpr int kHPrefetchItems = 1;  // kernel before this one drains, one lane per tile (more measured no better)
 static_assert(kHPrefetch * kHPrefetchItems <= 32, "one lane per prefetched tile");
@@ -63,6 +67,12 @@ struct TileMeta {
     long long new_row;  // cache row the new token is written to
     float sc;           // layer scale * log2(e)
     int pad2;
+};
+
+// Tensor maps over K and V with boxes of one head's slice by 1/kHHeights ... kHHeights/kHHeights of a
+// tile's rows: an item's last tile is fetched with the lowest box that holds its rows.
+struct HeadMaps {
+    CUtensorMap k[kHHeights], v[kHHeights];
 };
 
 struct HeadArgs {
@@ -182,8 +192,7 @@ template <> struct HVec<__nv_bfloat16> {
 // warp holds G = 32 / LPR rows at a time and a tile (8 KiB) is 16 such steps.
 template <typename T, int D>
 __global__ void __launch_bounds__((kHWarps + kHProducers) * 32, 1)
-decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                    const HeadArgs a)
+decode_heads_kernel(const __grid_constant__ HeadMaps maps, const HeadArgs a)
 {
     constexpr int VE = HVec<T>::VE;
     constexpr uint32_t SLICE = D * sizeof(T);
@@ -213,8 +222,11 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
 
     if (tid == 0) {
         s_abort = 0;
-        prefetch_map(&map_k);
-        prefetch_map(&map_v);
+#pragma unroll
+        for (int i = 0; i < kHHeights; ++i) {
+            prefetch_map(&maps.k[i]);
+            prefetch_map(&maps.v[i]);
+        }
         for (int i = 0; i < kHStages; ++i) {
             hbar_init(full + i, 1);
             hbar_init(empty + i, 1);
@@ -242,8 +254,8 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
             const long long off = a.row_offset[seg];
             const int cp = a.cap[seg];
             if (off >= 0 && off + cp <= a.total_cap_rows && t * TILE_ROWS < cp) {
-                tma_prefetch_2d(&map_k, h * D, (int)off + t * TILE_ROWS);
-                tma_prefetch_2d(&map_v, h * D, (int)off + t * TILE_ROWS);
+                tma_prefetch_2d(&maps.k[kHHeights - 1], h * D, (int)off + t * TILE_ROWS);
+                tma_prefetch_2d(&maps.v[kHHeights - 1], h * D, (int)off + t * TILE_ROWS);
             }
         }
     }
@@ -318,7 +330,9 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     m->item = item_seq;
                     m->seg = seg;
                     m->h = h;
-                    m->nrows = min(TILE_ROWS, ln - t * TILE_ROWS);
+                    const int nrows = min(TILE_ROWS, ln - t * TILE_ROWS);
+                    const int quarters = (nrows + TILE_ROWS / kHHeights - 1) / (TILE_ROWS / kHHeights);  // box height, in steps
+                    m->nrows = nrows;
                     m->flags = (last && append ? kFlagNew : 0) | (last ? kFlagItemLast : 0) |
                                (t + kHWarps >= tiles ? kFlagWarpLast : 0);
                     m->tiles = tiles;
@@ -326,13 +340,14 @@ decode_heads_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
                     m->slot_parity = slot_parity;
                     m->new_row = off + ln;
                     m->sc = s_scale[si];
-                    const uint32_t bytes = 2 * kHTile + SLICE + (last && append ? 2 * SLICE : 0u);
+                    const uint32_t bytes = 2 * (uint32_t)quarters * (kHTile / kHHeights) + SLICE + (last && append ? 2 * SLICE : 0u);
                     hbar_expect_tx(full + st, bytes);
                     const size_t hoff = ((size_t)seg * H + h) * SLICE;
-                    // rows past the segment's length (or past the cache: zero-filled) are masked by nrows
+                    // rows past the segment's length (fetched up to the box's height, zero-filled past the
+                    // cache, or left in the stage by its previous tile) are masked by nrows
                     const int row0 = (int)(off + (int64_t)t * TILE_ROWS);
-                    tma_load_2d(sb + HEAD, &map_k, full + st, h * D, row0);
-                    tma_load_2d(sb + HEAD + kHTile, &map_v, full + st, h * D, row0);
+                    tma_load_2d(sb + HEAD, &maps.k[quarters - 1], full + st, h * D, row0);
+                    tma_load_2d(sb + HEAD + kHTile, &maps.v[quarters - 1], full + st, h * D, row0);
                     hbulk_load(sb + 64, reinterpret_cast<const unsigned char *>(a.q) + hoff, SLICE, full + st);
                     if (last && append) {
                         hbulk_load(sb + 64 + SLICE, reinterpret_cast<const unsigned char *>(a.k_new) + hoff, SLICE, full + st);
@@ -593,7 +608,7 @@ bool make_cache_map(CUtensorMap *map, void *ptr, const pkv_shape *s, int64_t row
 }
 
 template <typename T, int D>
-int launch_heads(const CUtensorMap *maps, const HeadArgs &a, int grid, cudaStream_t st)
+int launch_heads(const HeadMaps &maps, const HeadArgs &a, int grid, cudaStream_t st)
 {
     static bool done[64] = {};
     constexpr uint32_t SLICE = D * sizeof(T);
@@ -603,7 +618,7 @@ int launch_heads(const CUtensorMap *maps, const HeadArgs &a, int grid, cudaStrea
     int rc = ensure_dynamic_smem((const void *)decode_heads_kernel<T, D>, 226 * 1024, done);
     if (rc != PKV_OK) return rc;
     if (smem > 226 * 1024) return -1;
-    cudaError_t e = launch_dependent(decode_heads_kernel<T, D>, dim3(grid), dim3((kHWarps + kHProducers) * 32), smem, st, maps[0], maps[1], a);
+    cudaError_t e = launch_dependent(decode_heads_kernel<T, D>, dim3(grid), dim3((kHWarps + kHProducers) * 32), smem, st, maps, a);
     if (e != cudaSuccess) {
         set_cuda_error(e, "decode_heads_kernel");
         return PKV_ERR_CUDA;
@@ -646,10 +661,44 @@ int launch_decode_heads(const pkv_shape *s, pkv_cache *c, const void *q, const v
     if ((int64_t)nact * H < 4 * (int64_t)sms || call_bytes > kHMaxCallBytes) return -1;
     const size_t es = esize(s);
     const int tile_rows = (int)(kHTile / ((size_t)D * es));
-    CUtensorMap maps[2];
-    if (!make_cache_map(&maps[0], c->k, s, c->total_cap_rows, tile_rows) ||
-        !make_cache_map(&maps[1], c->v, s, c->total_cap_rows, tile_rows))
-        return -1;
+    // The maps depend on the cache's buffers and shape alone: the last few sets are kept, so that a
+    // decode loop encodes them once.
+    struct MapKey {
+        void *k, *v;
+        int64_t rows;
+        int heads, dim, dtype;
+    };
+    struct MapEntry {
+        MapKey key;
+        HeadMaps maps;
+        bool used;
+    };
+    static std::mutex map_mutex;
+    static MapEntry map_cache[4];
+    static int map_next = 0;
+    const MapKey key{c->k, c->v, c->total_cap_rows, H, D, (int)s->dtype};
+    HeadMaps maps;
+    {
+        std::lock_guard<std::mutex> guard(map_mutex);
+        const MapEntry *hit = nullptr;
+        for (const MapEntry &e : map_cache)
+            if (e.used && e.key.k == key.k && e.key.v == key.v && e.key.rows == key.rows && e.key.heads == key.heads &&
+                e.key.dim == key.dim && e.key.dtype == key.dtype)
+                hit = &e;
+        if (hit) {
+            maps = hit->maps;
+        } else {
+            for (int i = 0; i < kHHeights; ++i)
+                if (!make_cache_map(&maps.k[i], c->k, s, c->total_cap_rows, tile_rows * (i + 1) / kHHeights) ||
+                    !make_cache_map(&maps.v[i], c->v, s, c->total_cap_rows, tile_rows * (i + 1) / kHHeights))
+                    return -1;
+            MapEntry &e = map_cache[map_next];
+            map_next = (map_next + 1) % 4;
+            e.key = key;
+            e.maps = maps;
+            e.used = true;
+        }
+    }
 
     static std::atomic<unsigned long long> g_token{
         0x9e3779b97f4a7c15ull ^ (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count()};
