@@ -81,8 +81,7 @@ DECODE_KERNELS = {
 def decode_path(w, sms):
     nact = w.B * w.L
     cap_rows = w.B * (min(w.budget_rows(), w.L * w.N) + w.L * w.T)       # as Session sizes the cache
-    call_bytes = 2.0 * cap_rows * w.H * w.D * w.esize
-    heads = w.D in (64, 128) and nact <= 256 and nact * w.H >= 4 * sms and call_bytes <= 768 * 2**20
+    heads = w.D in (64, 128) and nact <= 256 and nact * w.H >= 4 * sms and cap_rows // nact <= 1024
     return "heads" if heads else "stream"
 
 

@@ -53,7 +53,7 @@ static_assert(kHPrefetch * kHPrefetchItems <= 32, "one lane per prefetched tile"
 constexpr int kHSlots = 4;         // items whose partial results may be waiting for their last tile
 constexpr int kHMaxAct = 256;      // segments planned per call
 constexpr int kHMaxGrid = 256;
-constexpr double kHMaxCallBytes = 768.0 * 1024 * 1024;  // larger calls go to the row-split kernel
+constexpr int64_t kHMaxSegRows = 1024;  // mean capacity of a segment above which calls go to the row-split kernel
 constexpr uint32_t kHTile = 8192;  // bytes of one K (or V) tile: 16 rows per row group of a warp
 constexpr int kHProducers = 2;     // issuing threads (one per warp): stage s is always filled by producer s mod kHProducers
 static_assert(kHStages % kHProducers == 0, "a stage must keep its producer, which then sees each of its phases in turn");
@@ -652,13 +652,15 @@ int launch_decode_heads(const pkv_shape *s, pkv_cache *c, const void *q, const v
     }
     if (sms > kHMaxGrid) sms = kHMaxGrid;
     // Worth it while complete (segment, head) items balance over the SMs (at least four per SM)
-    // and the call is small enough for its fixed costs to matter.  Measured on 32 layers x 32
-    // heads of 128, 128-256 rows per segment: 16 % faster than the row-split kernel at batch 1
-    // (100 MB per call), 9 % at batch 2, 2 % at batch 4, equal at batch 6 (600 MB); on 128
-    // segments of 800-1800 rows (2.8 GB per call) 26 % slower, because whole 8 KiB rows stream
-    // better than head-wide boxes.  The call's bytes are bounded here by the cache's capacity.
-    const double call_bytes = 2.0 * (double)c->total_cap_rows * (double)H * D * (double)esize(s) * nl / s->layers;
-    if ((int64_t)nact * H < 4 * (int64_t)sms || call_bytes > kHMaxCallBytes) return -1;
+    // and the segments are short.  Measured on 32 layers x 32 heads of 128, 128-256 rows per
+    // segment, against the row-split kernel: 21.1 / 26.0 us per call at batch 1, 67.4 / 71.4 at
+    // batch 4, 129.3 / 134.0 at batch 8 (256 segments).  On 128 segments of a long prompt it wins
+    // while they hold under about 1000 rows (341 / 352 us) and loses beyond (561 / 502 us at 1800
+    // rows): the CTAs that work on neighbouring heads of a segment drift apart over a long item,
+    // and the 256-byte slices of a row are then fetched from DRAM one by one, while the row-split
+    // kernel always reads whole 8 KiB rows.  Lengths live on the device; the capacity bounds them.
+    const int64_t seg_rows = c->total_cap_rows / ((int64_t)s->batch * s->layers);
+    if ((int64_t)nact * H < 4 * (int64_t)sms || seg_rows > kHMaxSegRows) return -1;
     const size_t es = esize(s);
     const int tile_rows = (int)(kHTile / ((size_t)D * es));
     // The maps depend on the cache's buffers and shape alone: the last few sets are kept, so that a
