@@ -25,7 +25,8 @@
 // the prefetch below, against 21.95 for ten); two consumer warps per tile
 // (half the rows each) 22.4; an item's last, partial tile fetched in quarter-tile boxes 22.6 with
 // five producers, 27.3 with one; neighbouring heads fetched side by side in boxes twice as wide
-// and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7;
+// and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7 when a
+// producer thread waits for the atomic, 21.6 against 21.1 when a thirteenth warp does the claiming;
 // launched without the programmatic dependency 24.0 (all these with whole boxes for every tile;
 // choosing the last tile's box among four heights then took 21.95 to 21.15); an item's partial last tile read by its warp
 // straight from global memory (no bytes past the length) 27.0: plain loads queue behind the bulk
