@@ -372,7 +372,7 @@ def measure_workload(w, steps, warmup, dev, rank, world, sampler=None, with_lse=
     return res
 
 
-def workload_summary(w, m, hbm_peak, tf_peak):
+def workload_summary(w, m, hbm_peak, tf_peak, sms):
     """The figures of one configuration that the targets are stated on."""
     st = m["stage_ms"]
     dec_gbs = m["dec_bytes"] / (st["decode"] * 1e-3) / 1e9
@@ -381,7 +381,8 @@ def workload_summary(w, m, hbm_peak, tf_peak):
             "decode_pct_of_8tbs": 100 * dec_gbs / NOMINAL_HBM_GBS, "decode_us_per_call": 1e3 * st["decode"] / w.T,
             "compress_ms_per_prompt": compress_ms / w.B, "stages_ms": st,
             "score_tensor_util_vs_burst": m["causal_flop"] * 2 / (st["score"] * 1e-3) / (tf_peak * 1e12),
-            "tok_s": w.B * w.T / (sum(st.values()) * 1e-3), "prompts_interleaved": m["R"], "clocks": m["clocks"]}
+            "tok_s": w.B * w.T / (sum(st.values()) * 1e-3), "prompts_interleaved": m["R"], "clocks": m["clocks"],
+            "decode_kernel": DECODE_KERNELS[decode_path(w, sms)][0]}
 
 
 def run_ours(args):
@@ -428,15 +429,16 @@ def run_ours(args):
     # The other configurations, a few steps each (rank 0 of a one-GPU run only): the figures the
     # bandwidth and latency targets are stated on, measured in this same process.
     others = {}
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
     if world == 1 and not args.no_workloads and args.workload == "llava7b_b1":
-        others[w.name] = workload_summary(w, m, hbm_peak, tf_peak)
+        others[w.name] = workload_summary(w, m, hbm_peak, tf_peak, sms)
         for name in wl.ORDER:
             if name == w.name:
                 continue
             wo = wl.WORKLOADS[name]
             mo = measure_workload(wo, args.workload_steps, 3, dev, 0, 1, sampler)
             del mo["reps"], mo["pool"]
-            others[name] = workload_summary(wo, mo, hbm_peak, tf_peak)
+            others[name] = workload_summary(wo, mo, hbm_peak, tf_peak, sms)
             torch.cuda.empty_cache()
     clocks = m["clocks"]
     sampler.stop()
@@ -446,7 +448,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
     value = world * w.B * w.T / (step_ms_max * 1e-3)
-    path = decode_path(w, torch.cuda.get_device_properties(dev).multi_processor_count)
+    path = decode_path(w, sms)
     line = {
         "metric": "tok/s", "value": value, "unit": "tok/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True,
