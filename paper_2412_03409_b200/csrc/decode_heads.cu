@@ -28,7 +28,8 @@
 // and half as high 23.1; items claimed from a shared counter instead of dealt by position 24.7 when a
 // producer thread waits for the atomic, 21.6 against 21.1 when a thirteenth warp does the claiming;
 // a K and a V tile in one copy (a rank-3 map whose last stride is the distance between the two
-// buffers) 21.35 against 21.17;
+// buffers) 21.35 against 21.17; skipping, four at a time, the row steps past a short tile's rows
+// 22.1 against 21.2 (the branches cost the full tiles more than the short ones gain);
 // launched without the programmatic dependency 24.0 (all these with whole boxes for every tile;
 // choosing the last tile's box among four heights then took 21.95 to 21.15); an item's partial last tile read by its warp
 // straight from global memory (no bytes past the length) 27.0: plain loads queue behind the bulk
